@@ -1,0 +1,241 @@
+"""Pins for the fp64 CPU oracle: each test checks it against something other than
+itself -- a library routine (numpy matmul / argsort, torch SDPA), a pure-Python
+brute force that never sorts, a closed form, or an invariant the paper fixes."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import GATE_SOFTMAX_ALL, GATE_SOFTMAX_TOPK
+
+
+def _rand(shape, seed, scale=1.0):
+    return (np.random.default_rng(seed).standard_normal(shape) * scale).astype(np.float32)
+
+
+def _case(B=1, H=2, N=40, C=16, D=8, M=4, seed=0, bias=False):
+    X = _rand((B, N, C), seed)
+    Wr = _rand((C, M), seed + 1, 1.0 / math.sqrt(C))
+    b = _rand((M,), seed + 2) if bias else None
+    Q = _rand((B, H, N, D), seed + 3)
+    K = _rand((B, H, N, D), seed + 4)
+    V = _rand((B, H, N, D), seed + 5)
+    return X, Wr, b, Q, K, V
+
+
+def _softmax64(a):
+    a = a - a.max()
+    e = np.exp(a)
+    return e / e.sum()
+
+
+# ---------------------------------------------------------------- route (Eq. 2-4)
+@pytest.mark.parametrize("k,mode", [(1, GATE_SOFTMAX_ALL), (2, GATE_SOFTMAX_TOPK),
+                                    (2, GATE_SOFTMAX_ALL), (1, GATE_SOFTMAX_TOPK)])
+def test_route_against_library_matmul_and_argsort(k, mode):
+    X, Wr, b, *_ = _case(B=2, N=300, C=48, M=8, seed=3, bias=True)
+    gid, gate, logits = oracle.route(X, Wr, b, k, mode, want_logits=True)
+    ref = X.astype(np.float64) @ Wr.astype(np.float64) + b.astype(np.float64)
+    assert np.abs(logits - ref).max() < 1e-12
+    order = np.argsort(-ref, axis=-1, kind="stable")[..., :k]
+    assert np.array_equal(gid, order.astype(np.int32))
+    for bi in range(X.shape[0]):
+        for n in range(X.shape[1]):
+            p_all = _softmax64(ref[bi, n])
+            sel = order[bi, n]
+            want = p_all[sel] if mode == GATE_SOFTMAX_ALL else _softmax64(ref[bi, n, sel])
+            assert np.abs(gate[bi, n] - want).max() < 1e-14
+
+
+def test_route_tie_goes_to_lower_index():
+    X = _rand((1, 50, 8), 0)
+    w = _rand((8, 1), 1)
+    Wr = np.concatenate([w * 0.5, w, w, w * 0.25], axis=1)  # columns 1 and 2 tie exactly
+    gid, gate, _ = oracle.route(X, Wr, None, 2, GATE_SOFTMAX_TOPK)
+    lg = X[0].astype(np.float64) @ Wr.astype(np.float64)
+    for n in range(50):
+        if lg[n, 1] >= lg[n].max():  # the tied pair is on top
+            assert list(gid[0, n]) == [1, 2]
+            assert abs(gate[0, n, 0] - 0.5) < 1e-15 and abs(gate[0, n, 1] - 0.5) < 1e-15
+        else:
+            assert gid[0, n, 0] in (0, 3)
+
+
+def test_gate_identities():
+    X, Wr, b, *_ = _case(N=500, C=32, M=8, seed=7)
+    gid, gate, logits = oracle.route(X, Wr, None, 1, GATE_SOFTMAX_ALL, want_logits=True)
+    assert np.all(gate > 1.0 / 8 - 1e-15) and np.all(gate <= 1.0)      # top-1 of a softmax >= 1/M
+    gid2, gate2, _ = oracle.route(X, Wr, None, 2, GATE_SOFTMAX_TOPK)
+    assert np.abs(gate2.sum(-1) - 1.0).max() < 1e-15
+    assert np.all(gate2[..., 0] >= gate2[..., 1])
+    assert np.all(gid2[..., 0] != gid2[..., 1])
+    assert np.array_equal(gid2[..., 0], gid[..., 0])
+    # M = 1: the only gate is 1 in both modes
+    _, g1, _ = oracle.route(X, Wr[:, :1], None, 1, GATE_SOFTMAX_ALL)
+    assert np.all(g1 == 1.0)
+
+
+# ---------------------------------------------------------------- sort (Alg. 1 line 2)
+@pytest.mark.parametrize("k", [1, 2])
+def test_sort_against_stable_argsort(k):
+    rng = np.random.default_rng(5)
+    B, N, M = 3, 777, 6
+    if k == 1:
+        gid = rng.integers(0, M, size=(B, N, 1)).astype(np.int32)
+    else:
+        a = rng.integers(0, M, size=(B, N))
+        bb = (a + rng.integers(1, M, size=(B, N))) % M  # distinct second group
+        gid = np.stack([a, bb], -1).astype(np.int32)
+    if k == 1:
+        gid[gid == 4] = 3  # leave group 4 empty
+    offsets, perm, inv = oracle.sort(gid, M)
+    for b in range(B):
+        flat = gid[b].reshape(-1)
+        order = np.argsort(flat, kind="stable")            # library stable sort of assignments
+        assert np.array_equal(perm[b], (order // k).astype(np.int32))
+        counts = np.bincount(flat, minlength=M)
+        assert np.array_equal(offsets[b], np.concatenate([[0], np.cumsum(counts)]).astype(np.int32))
+        # inv is the inverse: position of assignment (n, j)
+        assert np.array_equal(order[inv[b].reshape(-1)], np.arange(N * k))
+        assert np.array_equal(perm[b][inv[b]], np.repeat(np.arange(N)[:, None], k, 1))
+
+
+# ---------------------------------------------------------------- attention (Eq. 1, 5)
+@pytest.mark.parametrize("mode", [GATE_SOFTMAX_ALL, GATE_SOFTMAX_TOPK])
+def test_m1_is_full_attention(mode):
+    X, Wr, _, Q, K, V = _case(B=2, H=3, N=65, C=16, D=16, M=1, seed=11)
+    scale = 1.0 / math.sqrt(16)
+    out = oracle.forward(X, Wr, None, Q, K, V, 1, mode, scale)
+    q, k_, v = (torch.from_numpy(t).double() for t in (Q, K, V))
+    ref = torch.nn.functional.scaled_dot_product_attention(q, k_, v, scale=scale).numpy()
+    assert np.abs(out["O"] - ref).max() < 1e-13
+    # and the textbook formula with numpy primitives
+    s = np.einsum("bhnd,bhmd->bhnm", Q.astype(np.float64), K.astype(np.float64)) * scale
+    p = np.exp(s - s.max(-1, keepdims=True))
+    p /= p.sum(-1, keepdims=True)
+    assert np.abs(out["O"] - p @ V.astype(np.float64)).max() < 1e-13
+    assert np.all(out["gate"] == 1.0)
+    assert np.array_equal(out["perm"][0], np.arange(65))
+
+
+def _brute_force(X, Wr, bias, Q, K, V, k, mode, scale):
+    """Definition of Eq. 2-5 with python loops: no sort, no offsets, no perm."""
+    B, N, C = X.shape
+    M = Wr.shape[1]
+    H, D = Q.shape[1], Q.shape[3]
+    O = np.zeros((B, H, N, D))
+    for b in range(B):
+        sel, gates = [], []
+        for n in range(N):
+            r = [sum(float(X[b, n, c]) * float(Wr[c, i]) for c in range(C)) +
+                 (float(bias[i]) if bias is not None else 0.0) for i in range(M)]
+            idx = sorted(range(M), key=lambda i: (-r[i], i))[:k]
+            pool = range(M) if mode == GATE_SOFTMAX_ALL else idx
+            mx = max(r)
+            Z = sum(math.exp(r[i] - mx) for i in pool)
+            sel.append(idx)
+            gates.append([math.exp(r[i] - mx) / Z for i in idx])
+        for h in range(H):
+            for n in range(N):
+                for j, g in enumerate(sel[n]):
+                    mem = [m for m in range(N) if g in sel[m]]
+                    a = np.array([float(np.dot(Q[b, h, n].astype(np.float64),
+                                               K[b, h, m].astype(np.float64))) * scale for m in mem])
+                    p = _softmax64(a)
+                    for w, m in zip(p, mem):
+                        O[b, h, n] += gates[n][j] * w * V[b, h, m].astype(np.float64)
+    return O
+
+
+@pytest.mark.parametrize("M,k,mode,bias", [(4, 1, GATE_SOFTMAX_ALL, False), (4, 2, GATE_SOFTMAX_TOPK, True),
+                                           (3, 2, GATE_SOFTMAX_ALL, False), (2, 1, GATE_SOFTMAX_TOPK, True),
+                                           (4, 4, GATE_SOFTMAX_TOPK, False)])
+def test_forward_against_brute_force(M, k, mode, bias):
+    X, Wr, b, Q, K, V = _case(B=2, H=2, N=37, C=8, D=8, M=M, seed=20 + M + k, bias=bias)
+    out = oracle.forward(X, Wr, b, Q, K, V, k, mode, 0.3)
+    ref = _brute_force(X, Wr, b, Q, K, V, k, mode, 0.3)
+    assert np.abs(out["O"] - ref).max() < 1e-12
+
+
+def test_attn_rows_matches_forward_rows():
+    X, Wr, b, Q, K, V = _case(B=2, H=2, N=50, M=4, seed=31)
+    out = oracle.forward(X, Wr, None, Q, K, V, 2, GATE_SOFTMAX_TOPK, 0.25)
+    rows = np.array([[0, 0, 0], [1, 1, 49], [0, 1, 17], [1, 0, 3]], np.int32)
+    got = oracle.attn_rows(Q, K, V, out["gid"], out["gate"], out["offsets"], out["perm"], 0.25, rows)
+    for r, (bi, h, n) in enumerate(rows):
+        assert np.array_equal(got[r], out["O"][bi, h, n])
+
+
+def test_groups_are_independent():
+    """Eq. 5: a token only sees the keys and values of its own group."""
+    X, Wr, _, Q, K, V = _case(N=120, M=4, seed=40)
+    base = oracle.forward(X, Wr, None, Q, K, V, 1, GATE_SOFTMAX_ALL, 0.35)
+    g = base["gid"][0, :, 0]
+    K2, V2 = K.copy(), V.copy()
+    K2[:, :, g == 2] += 3.0
+    V2[:, :, g == 2] *= -2.0
+    pert = oracle.forward(X, Wr, None, Q, K2, V2, 1, GATE_SOFTMAX_ALL, 0.35)
+    assert np.array_equal(base["O"][:, :, g != 2], pert["O"][:, :, g != 2])
+    assert np.abs(base["O"][:, :, g == 2] - pert["O"][:, :, g == 2]).max() > 1e-3
+
+
+def test_token_order_does_not_matter():
+    """Eq. 1 is a set function of the group's (k, v) rows: shuffling tokens shuffles outputs."""
+    X, Wr, _, Q, K, V = _case(N=90, M=3, seed=50)
+    sh = np.random.default_rng(1).permutation(90)
+    a = oracle.forward(X, Wr, None, Q, K, V, 2, GATE_SOFTMAX_TOPK, 0.35)
+    b = oracle.forward(X[:, sh], Wr, None, Q[:, :, sh], K[:, :, sh], V[:, :, sh], 2,
+                       GATE_SOFTMAX_TOPK, 0.35)
+    assert np.array_equal(a["gid"][:, sh], b["gid"])
+    assert np.abs(a["O"][:, :, sh] - b["O"]).max() < 1e-13
+
+
+def test_closed_forms():
+    X, Wr, _, Q, K, V = _case(N=100, M=4, D=8, seed=60)
+    r = oracle.route(X, Wr, None, 1, GATE_SOFTMAX_ALL)
+    g, gate = r[0][0, :, 0], r[1][0, :, 0]
+    # (a) all V rows of a group equal v_g  ->  output = gate * v_g exactly (weights sum to 1)
+    vg = _rand((4, 8), 61)
+    Vc = np.broadcast_to(vg[g][None, None], V.shape).copy()
+    out = oracle.forward(X, Wr, None, Q, K, Vc, 1, GATE_SOFTMAX_ALL, 0.5)["O"]
+    want = gate[:, None] * vg[g].astype(np.float64)
+    assert np.abs(out - want[None, None]).max() < 1e-14
+    # (b) Q = 0  ->  uniform weights: output = gate * mean of the group's V rows
+    out0 = oracle.forward(X, Wr, None, np.zeros_like(Q), K, V, 1, GATE_SOFTMAX_ALL, 0.5)["O"]
+    for h in range(Q.shape[1]):
+        for grp in range(4):
+            mean = V[0, h, g == grp].astype(np.float64).mean(0)
+            got = out0[0, h, g == grp] / gate[g == grp][:, None]
+            assert np.abs(got - mean).max() < 1e-13
+    # (c) scale = 0 gives the same uniform weights whatever Q is
+    outs = oracle.forward(X, Wr, None, Q, K, V, 1, GATE_SOFTMAX_ALL, 0.0)["O"]
+    assert np.abs(outs - out0).max() < 1e-13
+
+
+def test_empty_and_single_token_groups():
+    X, Wr, _, Q, K, V = _case(N=64, M=4, seed=70)
+    bias = np.array([0.0, -1e4, 0.0, 0.0], np.float32)      # group 1 never chosen
+    out = oracle.forward(X, Wr, bias, Q, K, V, 1, GATE_SOFTMAX_ALL, 0.5)
+    assert out["offsets"][0, 1] == out["offsets"][0, 2]
+    assert np.all(np.isfinite(out["O"]))
+    # force token 5 alone into group 1: its output is gate * its own V row
+    Xs = X.copy()
+    Wb = Wr.copy()
+    Xs[0, 5] = 0.0
+    Xs[0, 5, 0] = 100.0
+    Wb[0] = [0.0, 1000.0, 0.0, 0.0]
+    Xs[0, :5, 0] = 0.0
+    Xs[0, 6:, 0] = 0.0
+    out = oracle.forward(Xs, Wb, bias, Q, K, V, 1, GATE_SOFTMAX_ALL, 0.5)
+    assert out["gid"][0, 5, 0] == 1 and (out["gid"][0, :, 0] == 1).sum() == 1
+    want = out["gate"][0, 5, 0] * V[0, :, 5].astype(np.float64)
+    assert np.abs(out["O"][0, :, 5] - want).max() < 1e-15
+
+
+def test_balanced_flops_are_one_over_m():
+    """Sec. 3.2: cost drops to 1/M of full attention under uniform assignment."""
+    from paper_2510_18692_b200.inputs import useful_flops
+    N, M, H, D = 4096, 8, 2, 64
+    assert useful_flops([N // M] * M, H, D) == pytest.approx(useful_flops([N], H, D) / M)
