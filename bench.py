@@ -1,0 +1,374 @@
+#!/usr/bin/env python
+"""Benchmark of the MoGA routed group-attention forward on B200.
+
+One "step" is one pass of the whole hot path (route -> sort -> gather -> group
+attention -> gated unpermute) over one layer-sized batch of synthetic input, by
+default the minute-long 561,600-token context.  Prints ONE JSON line:
+effective TFLOP/s (useful FLOPs = H * sum_g 4 n_g^2 D of the run's actual group
+sizes), the per-stage breakdown, the roofline of the dominant kernel, the same
+metric end to end from host buffers, and the CPU oracle timed beside it.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl reference]
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs
+its own layer (weak scaling, no collective on the data path); time is the max
+over ranks and `value` the whole-job aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2510_18692_b200.inputs import CONFIGS, make_inputs, useful_flops  # noqa: E402
+
+METRIC = "MoGA fwd effective TFLOP/s (bf16)"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+KERNELS_PER_FORWARD = 8   # route, 3 sort kernels, gather, attention schedule, attention, unpermute
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+# ----------------------------------------------------------------------------- distributed glue
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), \
+        int(os.environ.get("WORLD_SIZE", 1))
+
+
+def aggregate(ms_local: float, units_local: float, device=None):
+    """Max of the per-rank times and sum of the per-rank work (all ranks get both)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return ms_local, units_local
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    u = torch.tensor([units_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def barrier_sync():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample(cfg, host, routing, target_s=12.0):
+    """Time the oracle, as it stands, on a bounded sample: routing of 1,024 tokens and
+    attention rows of head 0 (calibrated on 64 rows to fill about `target_s` seconds)."""
+    import oracle
+    gid, gate, offsets, perm = routing
+    rng = np.random.default_rng(0)
+    tok = np.sort(rng.choice(cfg.N, size=min(1024, cfg.N), replace=False))
+    t0 = time.perf_counter()
+    oracle.route(host["X"][:, tok], host["Wr"], host["bias"], cfg.k, cfg.gate_mode)
+    t_route = time.perf_counter() - t0
+    sizes = np.diff(offsets[0])
+
+    def run(nrows, seed):
+        r = np.random.default_rng(seed)
+        rows = np.stack([np.zeros(nrows, np.int32), np.zeros(nrows, np.int32),
+                         r.integers(0, cfg.N, nrows).astype(np.int32)], 1)
+        fl = sum(4.0 * sizes[g] * cfg.D for n in rows[:, 2] for g in gid[0, n])
+        t0 = time.perf_counter()
+        oracle.attn_rows(host["Q"], host["K"], host["V"], gid, gate, offsets, perm, cfg.scale, rows)
+        return time.perf_counter() - t0, fl
+
+    t_cal, fl_cal = run(64, 1)
+    nrows = int(max(64, min(200000, 64 * target_s / max(t_cal, 1e-4))))
+    t, fl = run(nrows, 2)
+    return dict(tflops=fl / t / 1e12, seconds=t, rows=nrows, flops=fl, route_tokens=len(tok),
+                route_seconds=t_route, cores=oracle.threads())
+
+
+def run_reference(args, cfg):
+    """--impl reference: the CPU oracle, as it stands, on a bounded sample of the workload."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return 0
+    import oracle
+    small = cfg.with_(H=1)
+    inp = make_inputs(small, device="cpu", heads=[0])
+    host = {k: (None if v is None else v.float().numpy()) for k, v in inp.items()}
+    gid, gate, _ = oracle.route(host["X"], host["Wr"], host["bias"], cfg.k, cfg.gate_mode)
+    offsets, perm, _ = oracle.sort(gid, cfg.M)
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    vals, secs, rows = [], [], 0
+    for i in range(args.warmup + args.steps):
+        r = oracle_sample(cfg, host, (gid, gate, offsets, perm), target_s=per_step)
+        if i >= args.warmup:
+            vals.append(r["tflops"])
+            secs.append(r["seconds"])
+            rows = r["rows"]
+    v = float(np.mean(vals))
+    sample = f"{rows} attention rows of head 0 per step (fp64 oracle, routing from the oracle)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(secs)),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": config_dict(cfg),
+        "cpu_baseline": {"value": v, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": v, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+    return 0
+
+
+def config_dict(cfg):
+    return {"workload": cfg.name, "B": cfg.B, "H": cfg.H, "N": cfg.N, "C": cfg.C, "D": cfg.D, "M": cfg.M,
+            "k": cfg.k, "gate_mode": "softmax_all" if cfg.gate_mode == 0 else "softmax_topk",
+            "l2": "inputs larger than L2 (no flush needed)"}
+
+
+# ----------------------------------------------------------------------------- GPU arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="minute_bf16", choices=sorted(CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = CONFIGS[args.config]
+    if args.impl == "reference":
+        return run_reference(args, cfg)
+
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+
+    from paper_2510_18692_b200 import build
+    build.build()
+    from paper_2510_18692_b200 import binding as mb   # raises if the CUDA library is missing
+
+    cfg = cfg.with_(seed=cfg.seed + 100 * rank)       # every rank works on its own layer
+    inp = make_inputs(cfg, device=dev)
+    sh = mb.make_shape(cfg)
+    ws = mb.alloc_workspace(mb.moga_workspace_bytes(sh), dev)
+    O = torch.empty_like(inp["Q"])
+    T = cfg.T
+    gid = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.int32, device=dev)
+    gate = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.float32, device=dev)
+    perm = torch.empty(cfg.B, T, dtype=torch.int32, device=dev)
+    inv = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.int32, device=dev)
+    offsets = torch.empty(cfg.B, cfg.M + 1, dtype=torch.int32, device=dev)
+
+    def step():
+        mb.moga_forward(sh, inp["X"], inp["Wr"], inp["bias"], inp["Q"], inp["K"], inp["V"], O, ws,
+                        gid, gate, perm, offsets)
+
+    for _ in range(args.warmup):
+        step()
+    code, detail = mb.moga_last_device_status(ws)
+    if code != 0:
+        raise RuntimeError(f"device status {code} detail {detail:#x} after warm-up")
+    sizes = np.diff(offsets.cpu().numpy(), axis=1)
+    flops = sum(useful_flops(sizes[b], cfg.H, cfg.D) for b in range(cfg.B))
+
+    clocks = ClockSampler(local_rank)
+    clocks.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    barrier_sync()
+    ev[0].record()
+    for _ in range(args.steps):
+        step()
+    ev[1].record()
+    barrier_sync()
+    ms_local = ev[0].elapsed_time(ev[1]) / args.steps
+
+    # per-stage breakdown through the stage entry points (same kernels, same data)
+    es = 2 if cfg.dtype == "bf16" else 4
+    Qp, Kp, Vp, Op = (torch.empty(cfg.B, cfg.H, T, cfg.D, dtype=inp["Q"].dtype, device=dev) for _ in range(4))
+    stage_names = ["route", "permute", "group_attn", "unpermute"]
+    stage_ms = {n: [] for n in stage_names}
+    for it in range(args.steps + 1):
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+        e[0].record()
+        mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], gid, gate, None)
+        e[1].record()
+        mb.moga_permute(sh, gid, inp["Q"], inp["K"], inp["V"], perm, inv, offsets, Qp, Kp, Vp, ws)
+        e[2].record()
+        mb.moga_group_attn(sh, Qp, Kp, Vp, offsets, Op, None, ws)
+        e[3].record()
+        mb.moga_unpermute(sh, Op, inv, gate, O)
+        e[4].record()
+        torch.cuda.synchronize()
+        if it > 0:
+            for i, n in enumerate(stage_names):
+                stage_ms[n].append(e[i].elapsed_time(e[i + 1]))
+    clk = clocks.stop()
+    del Qp, Kp, Vp, Op
+    stage = {n: float(np.mean(v)) for n, v in stage_ms.items()}
+
+    ms, total_flops = aggregate(ms_local, flops, dev)
+    value = total_flops / (ms * 1e-3) / 1e12
+    peaks = load_peaks()
+    attn_tflops = flops / (stage["group_attn"] * 1e-3) / 1e12
+    tok = cfg.B * cfg.N
+    bytes_alg = {
+        "route": tok * cfg.C * es + tok * cfg.k * 8,
+        "permute": 3 * (1 + cfg.k) * tok * cfg.H * cfg.D * es + tok * cfg.k * 12,
+        "unpermute": (cfg.k + 1) * tok * cfg.H * cfg.D * es + tok * cfg.k * 8,
+    }
+    stages_out = {n: {"ms": stage[n]} for n in stage_names}
+    for n, by in bytes_alg.items():
+        gbs = by / (stage[n] * 1e-3) / 1e9
+        stages_out[n].update({"GB/s": gbs, "frac_hbm": gbs / peaks["hbm_gbs"]})
+    stages_out["group_attn"].update({"TFLOP/s": attn_tflops,
+                                     "frac_tensor_burst": attn_tflops / peaks["bf16_tflops"]})
+    out = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic", "config": config_dict(cfg),
+        "ms_per_layer_head_batch": ms / (cfg.B * cfg.H), "useful_tflop_per_step": flops / 1e12,
+        "group_sizes": {"min": int(sizes.min()), "max": int(sizes.max()), "empty": int((sizes == 0).sum())},
+        "stages": stages_out, "gpu_launches": KERNELS_PER_FORWARD * args.steps, "clocks": clk,
+        "roofline": {"kernel": "moga_group_attn (tcgen05 varlen attention)", "bound": "tensor",
+                     "achieved": attn_tflops, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                     "frac": attn_tflops / peaks["bf16_tflops_sustained"],
+                     "peak_source": f"{peaks['source']} sustained bf16 GEMM", "traffic": None},
+    }
+
+    if rank == 0 and not args.no_e2e:
+        out["e2e"] = run_e2e(mb, cfg, sh, inp, ws, O, flops, args)
+    if rank == 0 and not args.no_cpu and world == 1:
+        host = {n: inp[n][:, :1].float().cpu().numpy() for n in ("Q", "K", "V")}
+        host.update(Wr=inp["Wr"].cpu().numpy(), X=_LazyRows(inp["X"]),
+                    bias=None if inp["bias"] is None else inp["bias"].cpu().numpy())
+        # the sampled rows use the GPU's routing (same protocol as the parity tests)
+        r = oracle_sample(cfg, host, (gid.cpu().numpy(), gate.double().cpu().numpy(),
+                                      offsets.cpu().numpy(), perm.cpu().numpy()))
+        out["cpu_baseline"] = {"value": r["tflops"], "unit": "TFLOP/s", "cores": r["cores"], "kind": "oracle",
+                               "sample": f"{r['rows']} attention rows of head 0 in {r['seconds']:.1f} s "
+                                         f"(plus routing of {r['route_tokens']} tokens in {r['route_seconds']:.2f} s)"}
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(out))
+    return 0
+
+
+class _LazyRows:
+    """Host view of a large device X that materialises only the indexed token rows."""
+
+    def __init__(self, X):
+        self.X = X
+        self.shape = tuple(X.shape)
+
+    def __getitem__(self, idx):
+        b, tok = idx
+        assert b == slice(None)
+        return self.X[:, torch.from_numpy(np.asarray(tok)).to(self.X.device)].float().cpu().numpy()
+
+
+def run_e2e(mb, cfg, sh, inp, ws, O, flops, args):
+    """Same step from pinned host buffers: H2D of X, Q, K, V and D2H of O inside the timing."""
+    names = ["X", "Q", "K", "V"]
+    try:
+        host = {n: torch.empty(inp[n].shape, dtype=inp[n].dtype, pin_memory=True) for n in names}
+        host_O = torch.empty(O.shape, dtype=O.dtype, pin_memory=True)
+    except RuntimeError as e:   # not enough lockable host memory on this machine
+        return {"value": None, "unit": "TFLOP/s", "error": f"pinned allocation failed: {e}"[:200]}
+    for n in names:
+        host[n].copy_(inp[n])
+    dev_in = {n: torch.empty_like(inp[n]) for n in names}
+    h2d = sum(host[n].numel() * host[n].element_size() for n in names)
+    d2h = host_O.numel() * host_O.element_size()
+    steps = max(1, min(args.steps, 3))
+
+    def step():
+        for n in names:
+            dev_in[n].copy_(host[n], non_blocking=True)
+        mb.moga_forward(sh, dev_in["X"], inp["Wr"], inp["bias"], dev_in["Q"], dev_in["K"], dev_in["V"], O, ws)
+        host_O.copy_(O, non_blocking=True)
+
+    step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    return {"value": flops / (ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms, "steps": steps,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,142 @@
+/*
+ * moga.h -- C ABI of the B200 (sm_100a) MoGA routed group-attention forward.
+ *
+ * The library implements the forward of Mixture-of-Groups Attention
+ * (Sec. 3.2, Eq. 2-5 and Alg. 1 of the paper): a linear router scores each
+ * token against M groups, the token joins its top-k groups with a softmax gate,
+ * tokens are listed group by group (stable counting sort), Q/K/V rows are
+ * gathered into that order, dense softmax attention runs inside every group, and
+ * the rows go back to token order multiplied by their gates.
+ *
+ * Conventions shared by every entry point
+ *  - Every data pointer is a DEVICE pointer owned by the caller, 16-byte aligned.
+ *    The library allocates and frees nothing; all scratch lives in the caller's
+ *    workspace `ws` (device memory, 256-byte aligned).
+ *  - `stream` is a cudaStream_t passed as void*.  Calls are asynchronous on that
+ *    stream and never synchronise the host, except moga_last_device_status.
+ *  - Errors are return codes only.  A non-OK code from argument checking means
+ *    nothing was launched.
+ *  - Layouts (row-major, last index fastest):
+ *      X       [B, N, C]        dtype          token features
+ *      Wr      [C, M]           float          router weight
+ *      bias    [M]              float          router bias, may be NULL
+ *      Q,K,V,O [B, H, N, D]     dtype          element strides q_stride_{b,h,n}; D contiguous.
+ *                                              All-zero strides mean contiguous [B,H,N,D];
+ *                                              [B,N,H,D] is expressed through the strides.
+ *      gid     [B, N, k]        int32          selected groups, descending logit
+ *      gate    [B, N, k]        float          gate of each selected group
+ *      logits  [B, N, M]        float          optional router scores
+ *      perm    [B, T]           int32          token index at each sorted position, T = N*k
+ *      inv     [B, N, k]        int32          sorted position of assignment (n, j)
+ *      offsets [B, M+1]         int32          group g owns positions [offsets[g], offsets[g+1])
+ *      Qp,Kp,Vp,Op [B, H, T, D] dtype          rows in sorted (group-major) order, contiguous
+ *      lse     [B, H, T]        float          optional log-sum-exp of the scaled scores
+ *  - Limits: 1 <= M <= 64, 1 <= k <= min(M, 8), D in {64, 128}, C a multiple of
+ *    16 bytes worth of elements, N*k < 2^31.  Outside them: MOGA_ERR_UNSUPPORTED.
+ */
+#ifndef MOGA_H_
+#define MOGA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MOGA_OK = 0,
+  MOGA_ERR_INVALID_ARG = 1, /* null / misaligned pointer, non-positive size, bad enum   */
+  MOGA_ERR_UNSUPPORTED = 2, /* valid request outside the limits above                   */
+  MOGA_ERR_WORKSPACE = 3,   /* ws is NULL or smaller than the entry point requires      */
+  MOGA_ERR_CUDA = 4,        /* a CUDA runtime/driver call or a launch failed            */
+  MOGA_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up (see status word)     */
+  MOGA_ERR_INTERNAL = 6     /* device-side consistency check failed (e.g. gid range)    */
+} moga_status;
+
+typedef enum { MOGA_F32 = 0, MOGA_BF16 = 1 } moga_dtype;
+
+typedef enum {
+  MOGA_GATE_SOFTMAX_ALL = 0, /* Eq. 3-5: gate = softmax over all M logits, at the pick  */
+  MOGA_GATE_SOFTMAX_TOPK = 1 /* gate = softmax over the k selected logits               */
+} moga_gate_mode;
+
+typedef struct {
+  int32_t B, N, H, C, D, M, k;
+  int32_t dtype;     /* moga_dtype of X, Q, K, V, O and the permuted buffers            */
+  int32_t gate_mode; /* moga_gate_mode                                                  */
+  float scale;       /* softmax scale of Eq. 1, e.g. 1/sqrt(D); passed, never inferred  */
+  int64_t q_stride_b, q_stride_h, q_stride_n; /* element strides of Q, K, V and O       */
+} moga_shape;
+
+/* Host-only helpers: no CUDA call is made. */
+
+/* Bytes of `ws` moga_forward needs for this shape (0 if the shape is invalid). */
+size_t moga_workspace_bytes(const moga_shape* s);
+/* Bytes of `ws` the stage entry points (route, permute, group_attn) need. */
+size_t moga_scratch_bytes(const moga_shape* s);
+const char* moga_status_string(moga_status st);
+
+/*
+ * Router, Eq. 2-4: r = X W_r (+ bias) accumulated in fp32, the k largest logits
+ * per token (ties to the lower group index), and their gates (gate_mode).
+ * Writes gid, gate and, if non-NULL, logits.  Needs no workspace (ws may be NULL).
+ */
+moga_status moga_route(const moga_shape* s, const void* X, const float* Wr, const float* bias,
+                       int32_t* gid, float* gate, float* logits, void* ws, size_t ws_bytes,
+                       void* stream);
+
+/*
+ * "permute" of Alg. 1 line 2.  Stable counting sort of the N*k assignments of each
+ * batch item by group (ascending token index inside a group): writes perm, inv,
+ * offsets.  If Qp, Kp and Vp are all non-NULL the rows of Q, K, V are gathered
+ * into sorted order as well; all three NULL computes the indices only (Q, K, V may
+ * then be NULL).  ws: at least moga_scratch_bytes.  A gid outside [0, M) raises
+ * MOGA_ERR_INTERNAL in the device status word and is clamped.
+ */
+moga_status moga_permute(const moga_shape* s, const int32_t* gid, const void* Q, const void* K,
+                         const void* V, int32_t* perm, int32_t* inv, int32_t* offsets, void* Qp,
+                         void* Kp, void* Vp, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Alg. 1 line 3 / Eq. 1 inside each group: for every (b, h, g),
+ * Op_g = softmax(Qp_g Kp_g^T * scale) Vp_g, non-causal, no mask but the group
+ * boundary.  bf16 runs on tcgen05 tensor cores (fp32 accumulate and softmax);
+ * fp32 runs on the fp32 ALUs.  lse may be NULL.  ws: at least moga_scratch_bytes.
+ * An empty group does no work; a 1-token group returns its own V row.
+ */
+moga_status moga_group_attn(const moga_shape* s, const void* Qp, const void* Kp, const void* Vp,
+                            const int32_t* offsets, void* Op, float* lse, void* ws,
+                            size_t ws_bytes, void* stream);
+
+/*
+ * "repermute" of Alg. 1 line 4 with the gate of Eq. 5:
+ * O[b,h,n,:] = sum_j gate[b,n,j] * Op[b,h,inv[b,n,j],:], summed in fp32 in slot
+ * order and rounded once.  No workspace.
+ */
+moga_status moga_unpermute(const moga_shape* s, const void* Op, const int32_t* inv,
+                           const float* gate, void* O, void* stream);
+
+/*
+ * The whole forward: route -> permute -> group_attn -> unpermute with the
+ * intermediates in ws (at least moga_workspace_bytes).  gid_out, gate_out,
+ * perm_out, offsets_out may each be NULL; when given they receive copies of the
+ * routing results.
+ */
+moga_status moga_forward(const moga_shape* s, const void* X, const float* Wr, const float* bias,
+                         const void* Q, const void* K, const void* V, void* O, int32_t* gid_out,
+                         float* gate_out, int32_t* perm_out, int32_t* offsets_out, void* ws,
+                         size_t ws_bytes, void* stream);
+
+/*
+ * Synchronises `stream`, reads the device status word kept at the start of ws and
+ * clears it.  MOGA_OK if no kernel reported a problem since the last read,
+ * otherwise the first code recorded (MOGA_ERR_TIMEOUT, MOGA_ERR_INTERNAL).
+ * `detail`, if non-NULL, receives a kernel-specific word saying where.
+ */
+moga_status moga_last_device_status(void* ws, void* stream, uint32_t* detail);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOGA_H_ */

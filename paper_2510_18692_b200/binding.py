@@ -1,0 +1,127 @@
+"""Thin ctypes binding of the C ABI in include/moga.h (argument marshalling only).
+
+Every function takes torch CUDA tensors (used purely as device memory), passes
+their pointers and the current stream to ``libmoga.so`` and raises ``MogaError``
+on a non-OK status.  No arithmetic of the method happens in Python, and there is
+no fallback: if the library is missing, importing this module fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from .inputs import MogaConfig
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "csrc", "libmoga.so")
+
+EXPORTS = ("moga_workspace_bytes", "moga_scratch_bytes", "moga_status_string", "moga_route",
+           "moga_permute", "moga_group_attn", "moga_unpermute", "moga_forward",
+           "moga_last_device_status")
+
+MOGA_F32, MOGA_BF16 = 0, 1
+STATUS_NAMES = {0: "MOGA_OK", 1: "MOGA_ERR_INVALID_ARG", 2: "MOGA_ERR_UNSUPPORTED",
+                3: "MOGA_ERR_WORKSPACE", 4: "MOGA_ERR_CUDA", 5: "MOGA_ERR_TIMEOUT",
+                6: "MOGA_ERR_INTERNAL"}
+
+
+class MogaShape(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("N", ctypes.c_int32), ("H", ctypes.c_int32),
+                ("C", ctypes.c_int32), ("D", ctypes.c_int32), ("M", ctypes.c_int32),
+                ("k", ctypes.c_int32), ("dtype", ctypes.c_int32), ("gate_mode", ctypes.c_int32),
+                ("scale", ctypes.c_float), ("q_stride_b", ctypes.c_int64),
+                ("q_stride_h", ctypes.c_int64), ("q_stride_n", ctypes.c_int64)]
+
+
+class MogaError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {STATUS_NAMES.get(code, code)} ({status_string(code)})")
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2510_18692_b200.build` "
+                      "(there is no CPU fallback)")
+lib = ctypes.CDLL(LIB_PATH)
+lib.moga_workspace_bytes.restype = ctypes.c_size_t
+lib.moga_scratch_bytes.restype = ctypes.c_size_t
+lib.moga_status_string.restype = ctypes.c_char_p
+for _n in EXPORTS[3:]:
+    getattr(lib, _n).restype = ctypes.c_int
+
+
+def status_string(code: int) -> str:
+    return lib.moga_status_string(ctypes.c_int(code)).decode()
+
+
+def make_shape(cfg: MogaConfig, strides=None, scale=None) -> MogaShape:
+    sb, sh, sn = strides if strides is not None else (0, 0, 0)
+    return MogaShape(cfg.B, cfg.N, cfg.H, cfg.C, cfg.D, cfg.M, cfg.k,
+                     MOGA_F32 if cfg.dtype == "f32" else MOGA_BF16, cfg.gate_mode,
+                     cfg.scale if scale is None else scale, sb, sh, sn)
+
+
+def _ptr(t):
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise MogaError(code, where)
+
+
+def moga_workspace_bytes(shape: MogaShape) -> int:
+    return int(lib.moga_workspace_bytes(ctypes.byref(shape)))
+
+
+def moga_scratch_bytes(shape: MogaShape) -> int:
+    return int(lib.moga_scratch_bytes(ctypes.byref(shape)))
+
+
+def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """Device bytes for ``ws`` (torch's allocator returns 512-byte aligned blocks)."""
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def moga_route(shape, X, Wr, bias, gid, gate, logits=None, ws=None):
+    _check(lib.moga_route(ctypes.byref(shape), _ptr(X), _ptr(Wr), _ptr(bias), _ptr(gid), _ptr(gate),
+                          _ptr(logits), _ptr(ws), ctypes.c_size_t(0 if ws is None else ws.numel()),
+                          _stream()), "moga_route")
+
+
+def moga_permute(shape, gid, Q, K, V, perm, inv, offsets, Qp, Kp, Vp, ws):
+    _check(lib.moga_permute(ctypes.byref(shape), _ptr(gid), _ptr(Q), _ptr(K), _ptr(V), _ptr(perm),
+                            _ptr(inv), _ptr(offsets), _ptr(Qp), _ptr(Kp), _ptr(Vp), _ptr(ws),
+                            ctypes.c_size_t(ws.numel()), _stream()), "moga_permute")
+
+
+def moga_group_attn(shape, Qp, Kp, Vp, offsets, Op, lse, ws):
+    _check(lib.moga_group_attn(ctypes.byref(shape), _ptr(Qp), _ptr(Kp), _ptr(Vp), _ptr(offsets),
+                               _ptr(Op), _ptr(lse), _ptr(ws), ctypes.c_size_t(ws.numel()),
+                               _stream()), "moga_group_attn")
+
+
+def moga_unpermute(shape, Op, inv, gate, O):
+    _check(lib.moga_unpermute(ctypes.byref(shape), _ptr(Op), _ptr(inv), _ptr(gate), _ptr(O),
+                              _stream()), "moga_unpermute")
+
+
+def moga_forward(shape, X, Wr, bias, Q, K, V, O, ws, gid_out=None, gate_out=None, perm_out=None,
+                 offsets_out=None):
+    _check(lib.moga_forward(ctypes.byref(shape), _ptr(X), _ptr(Wr), _ptr(bias), _ptr(Q), _ptr(K),
+                            _ptr(V), _ptr(O), _ptr(gid_out), _ptr(gate_out), _ptr(perm_out),
+                            _ptr(offsets_out), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()),
+           "moga_forward")
+
+
+def moga_last_device_status(ws):
+    """(status code, detail word) of the most recent call that used ``ws``; synchronises."""
+    detail = ctypes.c_uint32(0)
+    code = lib.moga_last_device_status(_ptr(ws), _stream(), ctypes.byref(detail))
+    return int(code), int(detail.value)

@@ -1,0 +1,196 @@
+// C ABI of libmoga.so: argument validation, workspace carving, stage launches.
+#include "moga_internal.cuh"
+
+using namespace moga;
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Shape checks shared by every entry point.  Sets *st and returns false on failure.
+bool check_shape(const moga_shape* s, moga_status* st) {
+  if (s == nullptr) { *st = MOGA_ERR_INVALID_ARG; return false; }
+  if (s->B < 1 || s->N < 0 || s->H < 1 || s->C < 1 || s->D < 1 || s->M < 1 || s->k < 1 ||
+      (s->dtype != MOGA_F32 && s->dtype != MOGA_BF16) ||
+      (s->gate_mode != MOGA_GATE_SOFTMAX_ALL && s->gate_mode != MOGA_GATE_SOFTMAX_TOPK) ||
+      !(s->scale == s->scale)) {
+    *st = MOGA_ERR_INVALID_ARG;
+    return false;
+  }
+  const int epv = 16 / (int)elem_size(s->dtype);
+  if (s->M > kMaxM || s->k > s->M || s->k > kMaxK || (s->D != 64 && s->D != 128) ||
+      (s->C % epv) != 0 || (long long)s->N * s->k >= (1ll << 31) || s->H > 65535 ||
+      s->B > 65535) {
+    *st = MOGA_ERR_UNSUPPORTED;
+    return false;
+  }
+  const bool any = s->q_stride_b || s->q_stride_h || s->q_stride_n;
+  if (any) {
+    if (s->q_stride_b < 0 || s->q_stride_h < 0 || s->q_stride_n < s->D ||
+        (s->q_stride_b % epv) || (s->q_stride_h % epv) || (s->q_stride_n % epv)) {
+      *st = MOGA_ERR_INVALID_ARG;
+      return false;
+    }
+  }
+  *st = MOGA_OK;
+  return true;
+}
+
+bool check_ws(void* ws, size_t have, size_t need, moga_status* st) {
+  if (ws == nullptr || have < need || (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1))) {
+    *st = MOGA_ERR_WORKSPACE;
+    return false;
+  }
+  return true;
+}
+
+moga_status clear_header(char* ws, const WsLayout& L, cudaStream_t st) {
+  MOGA_CUDA_OK(cudaMemsetAsync(ws + L.header, 0, 256, st));
+  return MOGA_OK;
+}
+
+#define PTR_OK(p) ((p) != nullptr && aligned16(p))
+
+}  // namespace
+
+extern "C" {
+
+size_t moga_workspace_bytes(const moga_shape* s) {
+  moga_status st;
+  if (!check_shape(s, &st)) return 0;
+  return ws_layout(*s).total;
+}
+
+size_t moga_scratch_bytes(const moga_shape* s) {
+  moga_status st;
+  if (!check_shape(s, &st)) return 0;
+  return ws_layout(*s).scratch_end;
+}
+
+const char* moga_status_string(moga_status st) {
+  switch (st) {
+    case MOGA_OK: return "ok";
+    case MOGA_ERR_INVALID_ARG: return "invalid argument";
+    case MOGA_ERR_UNSUPPORTED: return "unsupported shape or type";
+    case MOGA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case MOGA_ERR_CUDA: return "CUDA call failed";
+    case MOGA_ERR_TIMEOUT: return "device-side wait timed out";
+    case MOGA_ERR_INTERNAL: return "device-side consistency check failed";
+  }
+  return "unknown status";
+}
+
+moga_status moga_route(const moga_shape* s, const void* X, const float* Wr, const float* bias,
+                       int32_t* gid, float* gate, float* logits, void* ws, size_t ws_bytes,
+                       void* stream) {
+  (void)ws;
+  (void)ws_bytes;
+  moga_status st;
+  if (!check_shape(s, &st)) return st;
+  if (!PTR_OK(X) || !PTR_OK(Wr) || !PTR_OK(gid) || !PTR_OK(gate) ||
+      (bias != nullptr && !aligned16(bias)) || (logits != nullptr && !aligned16(logits)))
+    return MOGA_ERR_INVALID_ARG;
+  return launch_route(*s, X, Wr, bias, gid, gate, logits, static_cast<cudaStream_t>(stream));
+}
+
+moga_status moga_permute(const moga_shape* s, const int32_t* gid, const void* Q, const void* K,
+                         const void* V, int32_t* perm, int32_t* inv, int32_t* offsets, void* Qp,
+                         void* Kp, void* Vp, void* ws, size_t ws_bytes, void* stream) {
+  moga_status st;
+  if (!check_shape(s, &st)) return st;
+  if (!PTR_OK(gid) || !PTR_OK(perm) || !PTR_OK(inv) || !PTR_OK(offsets)) return MOGA_ERR_INVALID_ARG;
+  const int n_out = (Qp != nullptr) + (Kp != nullptr) + (Vp != nullptr);
+  if (n_out != 0 && n_out != 3) return MOGA_ERR_INVALID_ARG;
+  if (n_out == 3 && (!PTR_OK(Q) || !PTR_OK(K) || !PTR_OK(V) || !aligned16(Qp) || !aligned16(Kp) ||
+                     !aligned16(Vp)))
+    return MOGA_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(*s);
+  if (!check_ws(ws, ws_bytes, L.scratch_end, &st)) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  char* w = static_cast<char*>(ws);
+  if ((st = clear_header(w, L, cs)) != MOGA_OK) return st;
+  if ((st = launch_sort(*s, L, gid, perm, inv, offsets, w, cs)) != MOGA_OK) return st;
+  if (n_out == 3) return launch_gather(*s, perm, Q, K, V, Qp, Kp, Vp, cs);
+  return MOGA_OK;
+}
+
+moga_status moga_group_attn(const moga_shape* s, const void* Qp, const void* Kp, const void* Vp,
+                            const int32_t* offsets, void* Op, float* lse, void* ws,
+                            size_t ws_bytes, void* stream) {
+  moga_status st;
+  if (!check_shape(s, &st)) return st;
+  if (!PTR_OK(Qp) || !PTR_OK(Kp) || !PTR_OK(Vp) || !PTR_OK(offsets) || !PTR_OK(Op) ||
+      (lse != nullptr && !aligned16(lse)))
+    return MOGA_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(*s);
+  if (!check_ws(ws, ws_bytes, L.scratch_end, &st)) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  char* w = static_cast<char*>(ws);
+  if ((st = clear_header(w, L, cs)) != MOGA_OK) return st;
+  if (s->dtype == MOGA_F32)
+    return launch_attn_f32(*s, static_cast<const float*>(Qp), static_cast<const float*>(Kp),
+                           static_cast<const float*>(Vp), offsets, static_cast<float*>(Op), lse, cs);
+  return launch_attn_bf16(*s, L, Qp, Kp, Vp, offsets, Op, lse, w, cs);
+}
+
+moga_status moga_unpermute(const moga_shape* s, const void* Op, const int32_t* inv,
+                           const float* gate, void* O, void* stream) {
+  moga_status st;
+  if (!check_shape(s, &st)) return st;
+  if (!PTR_OK(Op) || !PTR_OK(inv) || !PTR_OK(gate) || !PTR_OK(O)) return MOGA_ERR_INVALID_ARG;
+  return launch_unpermute(*s, Op, inv, gate, O, static_cast<cudaStream_t>(stream));
+}
+
+moga_status moga_forward(const moga_shape* s, const void* X, const float* Wr, const float* bias,
+                         const void* Q, const void* K, const void* V, void* O, int32_t* gid_out,
+                         float* gate_out, int32_t* perm_out, int32_t* offsets_out, void* ws,
+                         size_t ws_bytes, void* stream) {
+  moga_status st;
+  if (!check_shape(s, &st)) return st;
+  if (!PTR_OK(X) || !PTR_OK(Wr) || !PTR_OK(Q) || !PTR_OK(K) || !PTR_OK(V) || !PTR_OK(O) ||
+      (bias != nullptr && !aligned16(bias)))
+    return MOGA_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(*s);
+  if (!check_ws(ws, ws_bytes, L.total, &st)) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  char* w = static_cast<char*>(ws);
+  int32_t* gid = reinterpret_cast<int32_t*>(w + L.gid);
+  float* gate = reinterpret_cast<float*>(w + L.gate);
+  int32_t* perm = reinterpret_cast<int32_t*>(w + L.perm);
+  int32_t* inv = reinterpret_cast<int32_t*>(w + L.inv);
+  int32_t* offsets = reinterpret_cast<int32_t*>(w + L.offsets);
+  void* Qp = w + L.Qp;
+  void* Kp = w + L.Kp;
+  void* Vp = w + L.Vp;
+  void* Op = w + L.Op;
+  if ((st = clear_header(w, L, cs)) != MOGA_OK) return st;
+  if ((st = launch_route(*s, X, Wr, bias, gid, gate, nullptr, cs)) != MOGA_OK) return st;
+  if ((st = launch_sort(*s, L, gid, perm, inv, offsets, w, cs)) != MOGA_OK) return st;
+  if ((st = launch_gather(*s, perm, Q, K, V, Qp, Kp, Vp, cs)) != MOGA_OK) return st;
+  if (s->dtype == MOGA_F32)
+    st = launch_attn_f32(*s, static_cast<const float*>(Qp), static_cast<const float*>(Kp),
+                         static_cast<const float*>(Vp), offsets, static_cast<float*>(Op), nullptr, cs);
+  else
+    st = launch_attn_bf16(*s, L, Qp, Kp, Vp, offsets, Op, nullptr, w, cs);
+  if (st != MOGA_OK) return st;
+  if ((st = launch_unpermute(*s, Op, inv, gate, O, cs)) != MOGA_OK) return st;
+  const size_t T = (size_t)s->N * s->k;
+  if (gid_out) MOGA_CUDA_OK(cudaMemcpyAsync(gid_out, gid, sizeof(int32_t) * s->B * T, cudaMemcpyDeviceToDevice, cs));
+  if (gate_out) MOGA_CUDA_OK(cudaMemcpyAsync(gate_out, gate, sizeof(float) * s->B * T, cudaMemcpyDeviceToDevice, cs));
+  if (perm_out) MOGA_CUDA_OK(cudaMemcpyAsync(perm_out, perm, sizeof(int32_t) * s->B * T, cudaMemcpyDeviceToDevice, cs));
+  if (offsets_out) MOGA_CUDA_OK(cudaMemcpyAsync(offsets_out, offsets, sizeof(int32_t) * s->B * (s->M + 1), cudaMemcpyDeviceToDevice, cs));
+  return MOGA_OK;
+}
+
+moga_status moga_last_device_status(void* ws, void* stream, uint32_t* detail) {
+  if (ws == nullptr) return MOGA_ERR_WORKSPACE;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  uint32_t words[2] = {0, 0};
+  MOGA_CUDA_OK(cudaMemcpyAsync(words, ws, sizeof(words), cudaMemcpyDeviceToHost, cs));
+  MOGA_CUDA_OK(cudaStreamSynchronize(cs));
+  if (detail) *detail = words[1];
+  if (words[0] != 0) MOGA_CUDA_OK(cudaMemsetAsync(ws, 0, 8, cs));
+  return words[0] <= MOGA_ERR_INTERNAL ? static_cast<moga_status>(words[0]) : MOGA_ERR_INTERNAL;
+}
+
+}  // extern "C"

@@ -1,0 +1,95 @@
+// Internal declarations shared by the kernels of libmoga.so (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/moga.h"
+
+namespace moga {
+
+// ---------------------------------------------------------------------------
+// Workspace layout.  The first 256 bytes are the header every stage shares:
+//   word 0: device status (moga_status), word 1: detail, word 2: attention work
+//   counter.  Scratch for the sort and the attention scheduler follows, then
+//   (moga_forward only) the intermediate tensors.
+// ---------------------------------------------------------------------------
+constexpr size_t kWsAlign = 256;
+constexpr int kSortChunk = 4096;   // assignments handled by one sort block
+constexpr int kMaxM = 64;
+constexpr int kMaxK = 8;
+
+struct WsLayout {
+  size_t header;      // 256 B
+  size_t sort_hist;   // int32 [B, nblk, M]   per-block histograms, then bases
+  size_t sched;       // int32 [B, 3, M+1]    attention schedule (order, tile prefix, ...)
+  size_t scratch_end; // == moga_scratch_bytes
+  size_t gid, gate, perm, inv, offsets;  // routing results
+  size_t Qp, Kp, Vp, Op;                 // permuted tensors
+  size_t total;       // == moga_workspace_bytes
+  int nblk;           // sort blocks per batch item
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline size_t elem_size(int dtype) { return dtype == MOGA_BF16 ? 2 : 4; }
+
+inline WsLayout ws_layout(const moga_shape& s) {
+  WsLayout L{};
+  size_t T = (size_t)s.N * s.k;
+  L.nblk = (int)((T + kSortChunk - 1) / kSortChunk);
+  if (L.nblk < 1) L.nblk = 1;
+  size_t off = 0;
+  L.header = off;      off = align_up(off + 256, kWsAlign);
+  L.sort_hist = off;   off = align_up(off + sizeof(int32_t) * (size_t)s.B * L.nblk * s.M, kWsAlign);
+  L.sched = off;       off = align_up(off + sizeof(int32_t) * (size_t)s.B * 4 * (s.M + 1) + 64, kWsAlign);
+  L.scratch_end = off;
+  L.gid = off;         off = align_up(off + sizeof(int32_t) * (size_t)s.B * T, kWsAlign);
+  L.gate = off;        off = align_up(off + sizeof(float) * (size_t)s.B * T, kWsAlign);
+  L.perm = off;        off = align_up(off + sizeof(int32_t) * (size_t)s.B * T, kWsAlign);
+  L.inv = off;         off = align_up(off + sizeof(int32_t) * (size_t)s.B * T, kWsAlign);
+  L.offsets = off;     off = align_up(off + sizeof(int32_t) * (size_t)s.B * (s.M + 1), kWsAlign);
+  size_t row = (size_t)s.B * s.H * T * s.D * elem_size(s.dtype);
+  L.Qp = off;          off = align_up(off + row, kWsAlign);
+  L.Kp = off;          off = align_up(off + row, kWsAlign);
+  L.Vp = off;          off = align_up(off + row, kWsAlign);
+  L.Op = off;          off = align_up(off + row, kWsAlign);
+  L.total = off;
+  return L;
+}
+
+struct Strides { long long b, h, n; };
+inline Strides qkv_strides(const moga_shape& s) {
+  if (s.q_stride_b == 0 && s.q_stride_h == 0 && s.q_stride_n == 0)
+    return {(long long)s.H * s.N * s.D, (long long)s.N * s.D, (long long)s.D};
+  return {s.q_stride_b, s.q_stride_h, s.q_stride_n};
+}
+
+// Device status word: the first non-zero code wins.
+__device__ __forceinline__ void report_status(uint32_t* header, uint32_t code, uint32_t detail) {
+  if (atomicCAS(header, 0u, code) == 0u) header[1] = detail;
+}
+
+// Stage launchers (each returns MOGA_OK or MOGA_ERR_CUDA; arguments already validated).
+moga_status launch_route(const moga_shape& s, const void* X, const float* Wr, const float* bias,
+                         int32_t* gid, float* gate, float* logits, cudaStream_t st);
+moga_status launch_sort(const moga_shape& s, const WsLayout& L, const int32_t* gid, int32_t* perm,
+                        int32_t* inv, int32_t* offsets, char* ws, cudaStream_t st);
+moga_status launch_gather(const moga_shape& s, const int32_t* perm, const void* Q, const void* K,
+                          const void* V, void* Qp, void* Kp, void* Vp, cudaStream_t st);
+moga_status launch_unpermute(const moga_shape& s, const void* Op, const int32_t* inv,
+                             const float* gate, void* O, cudaStream_t st);
+moga_status launch_attn_f32(const moga_shape& s, const float* Qp, const float* Kp, const float* Vp,
+                            const int32_t* offsets, float* Op, float* lse, cudaStream_t st);
+moga_status launch_attn_bf16(const moga_shape& s, const WsLayout& L, const void* Qp, const void* Kp,
+                             const void* Vp, const int32_t* offsets, void* Op, float* lse, char* ws,
+                             cudaStream_t st);
+
+#define MOGA_CUDA_OK(expr)                                   \
+  do {                                                       \
+    cudaError_t e__ = (expr);                                \
+    if (e__ != cudaSuccess) return MOGA_ERR_CUDA;            \
+  } while (0)
+
+}  // namespace moga

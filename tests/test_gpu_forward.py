@@ -1,0 +1,176 @@
+"""End-to-end parity of moga_forward against the fp64 oracle.
+
+Small cases are compared element by element with the full oracle forward; the
+paper-sized workloads (the ones bench.py times) are compared on sampled rows the
+oracle can compute one by one: routing on a token sample, the sort bit for bit,
+and attention rows that include the first and last row of every non-empty group
+and every row of the tiny groups."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from parity import check_output, check_routing, check_sort, to_np32
+from paper_2510_18692_b200.inputs import (CONFIGS, GATE_SOFTMAX_ALL, GATE_SOFTMAX_TOPK, MogaConfig,
+                                          make_inputs, torch_dtype)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mb():
+    from paper_2510_18692_b200 import build
+    build.build()
+    from paper_2510_18692_b200 import binding
+    return binding
+
+
+def run_forward(mb, cfg, inp, strides=None, O=None):
+    sh = mb.make_shape(cfg, strides=strides)
+    ws = mb.alloc_workspace(mb.moga_workspace_bytes(sh))
+    if O is None:
+        O = torch.empty_like(inp["Q"])
+    T = cfg.N * cfg.k
+    gid = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.int32, device="cuda")
+    gate = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.float32, device="cuda")
+    perm = torch.empty(cfg.B, T, dtype=torch.int32, device="cuda")
+    offsets = torch.empty(cfg.B, cfg.M + 1, dtype=torch.int32, device="cuda")
+    mb.moga_forward(sh, inp["X"], inp["Wr"], inp["bias"], inp["Q"], inp["K"], inp["V"], O, ws,
+                    gid, gate, perm, offsets)
+    assert mb.moga_last_device_status(ws) == (0, 0)
+    return O, gid, gate, perm, offsets
+
+
+def full_parity(mb, cfg, strides=None, layout_bnhd=False):
+    inp = make_inputs(cfg, device="cuda")
+    host = {k: to_np32(v) for k, v in inp.items()}
+    if layout_bnhd:
+        for n in ("Q", "K", "V"):
+            inp[n] = inp[n].permute(0, 2, 1, 3).contiguous()       # stored [B,N,H,D]
+        O = torch.empty_like(inp["Q"])
+        strides = (cfg.N * cfg.H * cfg.D, cfg.D, cfg.H * cfg.D)
+    else:
+        O = None
+    O, gid, gate, perm, offsets = run_forward(mb, cfg, inp, strides, O)
+    if layout_bnhd:
+        O = O.permute(0, 2, 1, 3)
+    o_gid, o_gate, o_logits = oracle.route(host["X"], host["Wr"], host["bias"], cfg.k, cfg.gate_mode, True)
+    flips = check_routing(gid, gate, o_logits, o_gid, o_gate, cfg.k)
+    o_off, o_perm, _ = oracle.sort(gid.cpu().numpy(), cfg.M)
+    assert np.array_equal(offsets.cpu().numpy(), o_off) and np.array_equal(perm.cpu().numpy(), o_perm)
+    want = oracle.attn_all(host["Q"], host["K"], host["V"], gid.cpu().numpy(),
+                           gate.double().cpu().numpy(), o_off, o_perm, cfg.scale)
+    if flips == 0:
+        # no near-tie was resolved differently: the fully independent oracle forward must agree too
+        ref = oracle.forward(host["X"], host["Wr"], host["bias"], host["Q"], host["K"], host["V"], cfg.k,
+                             cfg.gate_mode, cfg.scale)
+        assert np.array_equal(ref["perm"], o_perm)
+        assert np.abs(ref["O"] - want).max() <= 1e-5
+    return check_output(O.float().cpu().numpy(), want, cfg.dtype)
+
+
+def test_tiny_f32_config(mb):
+    full_parity(mb, CONFIGS["tiny_f32"])
+
+
+def test_tiny_f32_m1_is_full_attention(mb):
+    cfg = CONFIGS["tiny_f32"].with_(M=1)
+    inp = make_inputs(cfg, device="cuda")
+    O, gid, gate, perm, offsets = run_forward(mb, cfg, inp)
+    assert torch.all(gate == 1.0) and torch.all(gid == 0)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        inp["Q"].double().cpu(), inp["K"].double().cpu(), inp["V"].double().cpu(), scale=cfg.scale)
+    check_output(O.cpu().numpy(), ref.numpy(), "f32")
+
+
+SMALL = [
+    MogaConfig("s_bf16_top1", 1, 3, 3000, 256, 128, 8, 1, "bf16", GATE_SOFTMAX_ALL, 11),
+    MogaConfig("s_bf16_top2", 2, 2, 1500, 320, 128, 16, 2, "bf16", GATE_SOFTMAX_TOPK, 12),
+    MogaConfig("s_bf16_skew", 1, 2, 4000, 256, 128, 64, 2, "bf16", GATE_SOFTMAX_TOPK, 13, zipf_bias=2.0),
+    MogaConfig("s_bf16_d64", 1, 2, 1111, 128, 64, 4, 1, "bf16", GATE_SOFTMAX_ALL, 14),
+    MogaConfig("s_f32_top2", 2, 2, 700, 96, 128, 5, 2, "f32", GATE_SOFTMAX_TOPK, 15),
+    MogaConfig("s_bf16_m1", 1, 2, 1000, 128, 128, 1, 1, "bf16", GATE_SOFTMAX_ALL, 16),
+]
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=lambda c: c.name)
+def test_small_configs(mb, cfg):
+    full_parity(mb, cfg)
+
+
+def test_bnhd_layout(mb):
+    full_parity(mb, SMALL[0].with_(N=999), layout_bnhd=True)
+
+
+def test_forward_is_deterministic(mb):
+    cfg = SMALL[1]
+    inp = make_inputs(cfg, device="cuda")
+    a = run_forward(mb, cfg, inp)
+    b = run_forward(mb, cfg, inp)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+
+
+def sampled_parity(mb, cfg, n_route=4096, n_rows=2048, heads=(0,)):
+    """Paper-sized workload: GPU runs all of it, the oracle checks samples."""
+    heads = [h for h in heads if h < cfg.H] + ([cfg.H - 1] if cfg.H > 1 else [])
+    inp = make_inputs(cfg, device="cuda")
+    O, gid, gate, perm, offsets = run_forward(mb, cfg, inp)
+    rng = np.random.default_rng(cfg.seed)
+    # 1. routing on a token sample
+    for b in range(cfg.B):
+        idx = np.sort(rng.choice(cfg.N, size=min(n_route, cfg.N), replace=False))
+        tidx = torch.from_numpy(idx).cuda()
+        Xs = to_np32(inp["X"][b, tidx])[None]
+        o_gid, o_gate, o_logits = oracle.route(Xs, to_np32(inp["Wr"]), to_np32(inp["bias"]), cfg.k,
+                                               cfg.gate_mode, True)
+        check_routing(gid[b:b + 1, tidx], gate[b:b + 1, tidx], o_logits, o_gid, o_gate, cfg.k)
+    # 2. sort, bit for bit, on all assignments
+    gid_np = gid.cpu().numpy()
+    o_off, o_perm, o_inv = oracle.sort(gid_np, cfg.M)
+    assert np.array_equal(offsets.cpu().numpy(), o_off) and np.array_equal(perm.cpu().numpy(), o_perm)
+    # 3. attention rows: group boundaries, tiny groups, largest group, random rows
+    Qh, Kh, Vh = (to_np32(inp[n][:, heads]) for n in ("Q", "K", "V"))
+    rows = []
+    for b in range(cfg.B):
+        sizes = np.diff(o_off[b])
+        for g in range(cfg.M):
+            lo, hi = o_off[b, g], o_off[b, g + 1]
+            if hi == lo:
+                continue
+            pos = range(lo, hi) if hi - lo <= 4 else (lo, hi - 1, lo + (hi - lo) // 2)
+            rows += [(b, hi_, int(o_perm[b, p])) for p in pos for hi_ in range(len(heads))]
+        big = int(np.argmax(sizes))
+        pos = rng.integers(o_off[b, big], o_off[b, big + 1], size=8)
+        rows += [(b, 0, int(o_perm[b, p])) for p in pos]
+    rnd = max(0, n_rows - len(rows))
+    rows += list(zip(rng.integers(0, cfg.B, rnd).tolist(), rng.integers(0, len(heads), rnd).tolist(),
+                     rng.integers(0, cfg.N, rnd).tolist()))
+    rows = np.array(rows, np.int32)
+    want = oracle.attn_rows(Qh, Kh, Vh, gid_np, gate.double().cpu().numpy(), o_off, o_perm, cfg.scale, rows)
+    hmap = torch.tensor(heads, device="cuda")[torch.from_numpy(rows[:, 1]).long().cuda()]
+    got = O[torch.from_numpy(rows[:, 0]).long().cuda(), hmap, torch.from_numpy(rows[:, 2]).long().cuda()]
+    return check_output(got.float().cpu().numpy(), want, cfg.dtype)
+
+
+def test_clip_bf16_full_size(mb):
+    sampled_parity(mb, CONFIGS["clip_bf16"], heads=(0, 5))
+
+
+def test_minute_bf16_full_size_sampled(mb):
+    """The workload bench.py times (561,600 tokens), same launch configuration."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 80 * 2**30:
+        pytest.skip("needs ~70 GB of device memory")
+    sampled_parity(mb, CONFIGS["minute_bf16"], n_rows=1536)
+
+
+def test_multishot_bf16_full_size_sampled(mb):
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60 * 2**30:
+        pytest.skip("needs ~50 GB of device memory")
+    sampled_parity(mb, CONFIGS["multishot_bf16"], n_rows=1536)
+
+
+def test_skew_bf16_full_size_sampled(mb):
+    sampled_parity(mb, CONFIGS["skew_bf16"], n_rows=768)
