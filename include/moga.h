@@ -65,7 +65,7 @@ typedef struct {
   int32_t B, N, H, C, D, M, k;
   int32_t dtype;     /* moga_dtype of X, Q, K, V, O and the permuted buffers            */
   int32_t gate_mode; /* moga_gate_mode                                                  */
-  float scale;       /* softmax scale of Eq. 1, e.g. 1/sqrt(D); passed, never inferred  */
+  float scale;       /* softmax scale of Eq. 1, e.g. 1/sqrt(D); finite, >= 0; never inferred */
   int64_t q_stride_b, q_stride_h, q_stride_n; /* element strides of Q, K, V and O       */
 } moga_shape;
 
@@ -130,8 +130,9 @@ moga_status moga_forward(const moga_shape* s, const void* X, const float* Wr, co
 
 /*
  * Synchronises `stream`, reads the device status word kept at the start of ws and
- * clears it.  MOGA_OK if no kernel reported a problem since the last read,
- * otherwise the first code recorded (MOGA_ERR_TIMEOUT, MOGA_ERR_INTERNAL).
+ * clears it.  Every permute / group_attn / forward call resets the word when it
+ * starts, so the result describes the most recent such call on this ws: MOGA_OK,
+ * or the first problem a kernel recorded (MOGA_ERR_TIMEOUT, MOGA_ERR_INTERNAL).
  * `detail`, if non-NULL, receives a kernel-specific word saying where.
  */
 moga_status moga_last_device_status(void* ws, void* stream, uint32_t* detail);

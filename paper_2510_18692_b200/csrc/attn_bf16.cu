@@ -1,8 +1,627 @@
-// placeholder until the tcgen05 kernel lands
+// bf16 per-group attention (Eq. 1 inside each group, Alg. 1 line 3) on tcgen05 tensor cores.
+//
+// One persistent CTA per SM walks a cost-ordered list of work items.  An item is
+// (batch, head, group, block of 256 query rows): two 128-row Q tiles (A and B) that
+// share every K/V tile of the group, so the tensor pipe works on one tile while the
+// other tile's softmax runs.
+//
+//   warp 0      TMA producer: Q tiles and a ring of K / V tiles, 128B-swizzled,
+//               each signalled through an mbarrier (no multicast).
+//   warp 1      MMA issuer (one lane): S = Q K^T into TMEM, O += P V with P read
+//               from TMEM; owns the TMEM allocation.
+//   warps 4-7   softmax of tile A, one thread per query row; warps 8-11 tile B.
+//               Online softmax in the log2 domain with a lazily updated maximum:
+//               O is rescaled (in TMEM, by the same warps) only when the row
+//               maximum grew by more than 2^8.  They also run the epilogue:
+//               O / l -> bf16 -> shared memory -> coalesced, row-predicated stores.
+//
+// TMEM (512 columns): S_A [0,128) S_B [128,256) O_A [256,256+D) O_B [384,384+D);
+// P (bf16, two per column) overwrites the first 64 columns of its S tile.
+// Every mbarrier wait is bounded: on expiry the CTA records MOGA_ERR_TIMEOUT in the
+// workspace status word, all roles leave their loops, and TMEM is released.
+#include <cuda.h>
+
 #include "moga_internal.cuh"
+
 namespace moga {
-moga_status launch_attn_bf16(const moga_shape&, const WsLayout&, const void*, const void*,
-                             const void*, const int32_t*, void*, float*, char*, cudaStream_t) {
-  return MOGA_ERR_UNSUPPORTED;
+namespace {
+
+constexpr int kThreads = 384;
+constexpr int kTileM = 128;       // query rows per tile
+constexpr int kTileN = 128;       // keys per K/V tile
+constexpr int kQBlock = 2 * kTileM;
+constexpr uint64_t kWaitLimitNs = 4000000000ull;  // 4 s: far above any legitimate wait
+
+// ----------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
+                                            int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  lbo/sbo in bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// kind::f16 instruction descriptor: bf16 x bf16 -> f32, A K-major, B K-major or MN-major.
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
+         ((uint32_t)(M >> 4) << 24);
+}
+
+// ----------------------------------------------------------------------------- schedule
+// order[b*M + r]  : group with the r-th largest size in batch item b
+// prefix[b*M + r] : number of work items before (b, r); prefix[B*M] = total
+__global__ void attn_schedule_kernel(const int32_t* __restrict__ offsets, int32_t* __restrict__ order,
+                                     int32_t* __restrict__ prefix, int B, int M, int H) {
+  for (int idx = threadIdx.x; idx < B * M; idx += blockDim.x) {
+    const int b = idx / M, g = idx % M;
+    const int32_t* off = offsets + (size_t)b * (M + 1);
+    const int n = off[g + 1] - off[g];
+    int r = 0;
+    for (int o = 0; o < M; ++o) {
+      const int no = off[o + 1] - off[o];
+      r += (no > n) || (no == n && o < g);
+    }
+    order[b * M + r] = g;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int acc = 0;
+    for (int idx = 0; idx < B * M; ++idx) {
+      const int b = idx / M;
+      const int32_t* off = offsets + (size_t)b * (M + 1);
+      const int g = order[idx];
+      const int n = off[g + 1] - off[g];
+      prefix[idx] = acc;
+      acc += ((n + kQBlock - 1) / kQBlock) * H;
+    }
+    prefix[B * M] = acc;
+  }
+}
+
+struct Item {
+  int bh;        // b * H + h
+  int row0;      // first sorted position of the query block
+  int lo, hi;    // the group's range of sorted positions
+};
+
+__device__ __forceinline__ Item decode_item(int w, const int32_t* __restrict__ offsets,
+                                            const int32_t* __restrict__ order,
+                                            const int32_t* __restrict__ prefix, int BM, int M, int H) {
+  int lo = 0, hi = BM;           // largest idx with prefix[idx] <= w
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (prefix[mid] <= w) lo = mid; else hi = mid;
+  }
+  const int b = lo / M;
+  const int g = order[lo];
+  const int32_t* off = offsets + (size_t)b * (M + 1);
+  Item it;
+  it.lo = off[g];
+  it.hi = off[g + 1];
+  const int nqb = (it.hi - it.lo + kQBlock - 1) / kQBlock;
+  const int local = w - prefix[lo];
+  const int h = local / nqb, qb = local % nqb;
+  it.bh = b * H + h;
+  it.row0 = it.lo + qb * kQBlock;
+  return it;
+}
+
+// ----------------------------------------------------------------------------- the kernel
+template <int D>
+struct Cfg {
+  static constexpr int NS = (D == 128) ? 2 : 4;           // K and V ring depth
+  static constexpr int kBoxes = D / 64;                   // 64-column TMA boxes per tile
+  static constexpr int kBoxBytes = kTileM * 128;          // 128 rows x 128 bytes
+  static constexpr int kTileBytes = kBoxes * kBoxBytes;
+  static constexpr int kSmemQ = 0;
+  static constexpr int kSmemK = 2 * kTileBytes;
+  static constexpr int kSmemV = kSmemK + NS * kTileBytes;
+  static constexpr int kSmemBar = kSmemV + NS * kTileBytes;
+  static constexpr int kNumBars = 2 + 2 + 4 * NS + 2 + 2 + 2 + 2 + 2;
+  static constexpr int kSmemTotal = kSmemBar + 8 * kNumBars + 16;
+  static constexpr int kDynSmem = kSmemTotal + 1024;      // slack for 1024-byte alignment
+};
+
+struct Shared {   // indices into the mbarrier array
+  int q_full, q_empty, k_full, k_empty, v_full, v_empty, s_full, p_full, o_full, o_empty;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                 const __grid_constant__ CUtensorMap mapV, const int32_t* __restrict__ offsets,
+                 const int32_t* __restrict__ order, const int32_t* __restrict__ prefix,
+                 __nv_bfloat16* __restrict__ Op, float* __restrict__ lse, uint32_t* header, int T, int H,
+                 int M, int BM, float scale_log2, float scale) {
+  using C = Cfg<D>;
+  constexpr int NS = C::NS;
+  extern __shared__ unsigned char smem_raw[];
+  // 128B-swizzled tiles need 1024-byte aligned bases
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* smem = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t sQ = base + C::kSmemQ, sK = base + C::kSmemK, sV = base + C::kSmemV;
+  const uint32_t bars = base + C::kSmemBar;
+  constexpr int Q_FULL = 0, Q_EMPTY = 2, K_FULL = 4, K_EMPTY = 4 + NS, V_FULL = 4 + 2 * NS,
+                V_EMPTY = 4 + 3 * NS, S_FULL = 4 + 4 * NS, P_FULL = S_FULL + 2, O_FULL = S_FULL + 4,
+                O_EMPTY = S_FULL + 6, STG_FULL = S_FULL + 8;
+  auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + C::kSmemBar + 8 * C::kNumBars);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total_items = prefix[BM];
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(Q_FULL + i), 1);
+      mbar_init(bar(Q_EMPTY + i), kTileM);
+      mbar_init(bar(S_FULL + i), 1);
+      mbar_init(bar(P_FULL + i), kTileM);
+      mbar_init(bar(O_FULL + i), 1);
+      mbar_init(bar(O_EMPTY + i), kTileM);
+      mbar_init(bar(STG_FULL + i), kTileM);
+    }
+    for (int i = 0; i < NS; ++i) {
+      mbar_init(bar(K_FULL + i), 1);
+      mbar_init(bar(K_EMPTY + i), 1);
+      mbar_init(bar(V_FULL + i), 1);
+      mbar_init(bar(V_EMPTY + i), 1);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32((const void*)tmem_slot)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  // Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
+  auto wait = [&](int idx, uint32_t parity, uint32_t where) -> bool {
+    const uint32_t b = bar(idx);
+    if (mbar_try_wait(b, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(b, parity)) {
+      if ((++spins & 255u) == 0) {
+        if (*abort_flag) return false;
+        if (global_timer_ns() - t0 > kWaitLimitNs) {
+          *abort_flag = 1;
+          report_status(header, MOGA_ERR_TIMEOUT, (where << 24) | ((uint32_t)blockIdx.x << 8) | (uint32_t)idx);
+          return false;
+        }
+      }
+    }
+    return true;
+  };
+
+  if (warp == 0) {
+    // ===================================================================== TMA producer
+    if (lane == 0) {
+      uint32_t nq[2] = {0, 0}, nkv = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
+        const Item it = decode_item(w, offsets, order, prefix, BM, M, H);
+        const int ntiles = (it.hi - it.lo + kTileN - 1) / kTileN;
+        const bool validB = it.row0 + kTileM < it.hi;
+        for (int x = 0; x < (validB ? 2 : 1) && ok; ++x) {
+          ok = wait(Q_EMPTY + x, (nq[x] & 1u) ^ 1u, 1);
+          if (!ok) break;
+          mbar_expect_tx(bar(Q_FULL + x), C::kTileBytes);
+#pragma unroll
+          for (int bx = 0; bx < C::kBoxes; ++bx)
+            tma_load_3d(sQ + x * C::kTileBytes + bx * C::kBoxBytes, &mapQ, bar(Q_FULL + x), bx * 64,
+                        it.row0 + x * kTileM, it.bh);
+          ++nq[x];
+        }
+        for (int j = 0; j < ntiles && ok; ++j) {
+          const int s = nkv % NS;
+          const uint32_t ph = ((nkv / NS) & 1u) ^ 1u;
+          ok = wait(K_EMPTY + s, ph, 2);
+          if (!ok) break;
+          mbar_expect_tx(bar(K_FULL + s), C::kTileBytes);
+#pragma unroll
+          for (int bx = 0; bx < C::kBoxes; ++bx)
+            tma_load_3d(sK + s * C::kTileBytes + bx * C::kBoxBytes, &mapK, bar(K_FULL + s), bx * 64,
+                        it.lo + j * kTileN, it.bh);
+          ok = wait(V_EMPTY + s, ph, 3);
+          if (!ok) break;
+          mbar_expect_tx(bar(V_FULL + s), C::kTileBytes);
+#pragma unroll
+          for (int bx = 0; bx < C::kBoxes; ++bx)
+            tma_load_3d(sV + s * C::kTileBytes + bx * C::kBoxBytes, &mapV, bar(V_FULL + s), bx * 64,
+                        it.lo + j * kTileN, it.bh);
+          ++nkv;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ===================================================================== MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = instr_desc(kTileM, kTileN, false);
+      constexpr uint32_t idesc_pv = instr_desc(kTileM, D, true);
+      uint32_t nq[2] = {0, 0}, ns[2] = {0, 0}, np[2] = {0, 0}, no[2] = {0, 0}, nk = 0, nv = 0;
+      bool ok = true;
+      // S_x = Q_x K^T for the K tile in ring slot s
+      auto issue_qk = [&](int x, int s) {
+        const uint32_t qa = sQ + x * C::kTileBytes, kb = sK + s * C::kTileBytes;
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t o = (kk / 4) * C::kBoxBytes + (kk % 4) * 32;
+          mma_ss(tmem + x * kTileN, smem_desc(qa + o, 16, 1024), smem_desc(kb + o, 16, 1024), idesc_qk,
+                 kk > 0);
+        }
+      };
+      // O_x (+)= P_x V for the V tile in ring slot s
+      auto issue_pv = [&](int x, int s, bool accumulate) {
+        const uint32_t vb = sV + s * C::kTileBytes;
+#pragma unroll
+        for (int kk = 0; kk < kTileN / 16; ++kk)
+          mma_ts(tmem + 256 + x * 128, tmem + x * kTileN + kk * 8,
+                 smem_desc(vb + kk * 2048, C::kBoxBytes, 1024), idesc_pv, (accumulate || kk > 0) ? 1u : 0u);
+      };
+      for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
+        const Item it = decode_item(w, offsets, order, prefix, BM, M, H);
+        const int ntiles = (it.hi - it.lo + kTileN - 1) / kTileN;
+        const int nx = (it.row0 + kTileM < it.hi) ? 2 : 1;
+        // first S tiles
+        for (int x = 0; x < nx && ok; ++x) {
+          ok = wait(Q_FULL + x, nq[x] & 1u, 4);
+          ++nq[x];
+        }
+        if (!ok) break;
+        ok = wait(K_FULL + nk % NS, (nk / NS) & 1u, 5);
+        if (!ok) break;
+        tc_fence_after();
+        for (int x = 0; x < nx; ++x) {
+          issue_qk(x, nk % NS);
+          tc_commit(bar(S_FULL + x));
+        }
+        tc_commit(bar(K_EMPTY + nk % NS));
+        ++nk;
+        for (int j = 0; j < ntiles && ok; ++j) {
+          ok = wait(V_FULL + nv % NS, (nv / NS) & 1u, 6);
+          if (!ok) break;
+          const bool more = j + 1 < ntiles;
+          if (more) {
+            ok = wait(K_FULL + nk % NS, (nk / NS) & 1u, 7);
+            if (!ok) break;
+          }
+          for (int x = 0; x < nx && ok; ++x) {
+            ok = wait(P_FULL + x, np[x] & 1u, 8);
+            if (!ok) break;
+            ++np[x];
+            if (j == 0) {
+              ok = wait(O_EMPTY + x, (no[x] & 1u) ^ 1u, 9);
+              if (!ok) break;
+              ++no[x];
+            }
+            tc_fence_after();
+            issue_pv(x, nv % NS, j > 0);
+            if (more) {
+              issue_qk(x, nk % NS);
+              tc_commit(bar(S_FULL + x));
+            } else {
+              tc_commit(bar(O_FULL + x));
+            }
+          }
+          if (!ok) break;
+          tc_commit(bar(V_EMPTY + nv % NS));
+          ++nv;
+          if (more) {
+            tc_commit(bar(K_EMPTY + nk % NS));
+            ++nk;
+          }
+        }
+      }
+      (void)ns;
+    }
+  } else if (warp >= 4) {
+    // ===================================================================== softmax + epilogue
+    const int x = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
+    const int q = warp & 3;                        // TMEM lane quarter of this warp
+    const int r = q * 32 + lane;                   // row inside the tile
+    const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+    const uint32_t tS = tmem + lane_off + x * kTileN;
+    const uint32_t tO = tmem + lane_off + 256 + x * 128;
+    unsigned char* stage = smem + C::kSmemQ + x * C::kTileBytes;    // O staging reuses the Q tile
+    uint32_t n_s = 0, n_o = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
+      const Item it = decode_item(w, offsets, order, prefix, BM, M, H);
+      if (x == 1 && !(it.row0 + kTileM < it.hi)) continue;
+      const int ntiles = (it.hi - it.lo + kTileN - 1) / kTileN;
+      const int tile_row0 = it.row0 + x * kTileM;
+      float m = -INFINITY, l = 0.f;
+      for (int j = 0; j < ntiles && ok; ++j) {
+        ok = wait(S_FULL + x, n_s & 1u, 10);
+        if (!ok) break;
+        ++n_s;
+        tc_fence_after();
+        uint32_t sreg[128];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
+        tmem_wait_ld();
+        const int ncols = it.hi - it.lo - j * kTileN;     // valid keys in this tile (may exceed 128)
+        if (ncols < kTileN) {
+#pragma unroll
+          for (int c = 0; c < 128; ++c)
+            if (c >= ncols) sreg[c] = 0xff800000u;        // -inf
+        }
+        float mt = __uint_as_float(sreg[0]);
+#pragma unroll
+        for (int c = 1; c < 128; ++c) mt = fmaxf(mt, __uint_as_float(sreg[c]));
+        const float m_new = fmaxf(m, mt);
+        // keep the old maximum unless it is stale by more than 2^8 somewhere in this warp
+        const bool grow = j == 0 || (m_new - m) * scale_log2 > 8.0f;
+        const bool rescale = __any_sync(0xffffffffu, grow);
+        float alpha = 1.f;
+        if (rescale) {
+          alpha = j == 0 ? 0.f : ex2((m - m_new) * scale_log2);
+          m = m_new;
+        }
+        const float neg_m = -m * scale_log2;
+        float lsum = 0.f;
+        uint32_t preg[64];
+#pragma unroll
+        for (int c = 0; c < 64; ++c) {
+          const float p0 = ex2(fmaf(__uint_as_float(sreg[2 * c]), scale_log2, neg_m));
+          const float p1 = ex2(fmaf(__uint_as_float(sreg[2 * c + 1]), scale_log2, neg_m));
+          lsum += p0 + p1;
+          __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+          preg[c] = *reinterpret_cast<uint32_t*>(&pk);
+        }
+        l = l * alpha + lsum;
+        tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&preg[0]));
+        tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&preg[32]));
+        if (rescale && j > 0) {
+          // the S tile arriving implies the previous P V has completed: O is stable
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t oreg[32];
+            tmem_ld32(tO + c * 32, oreg);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) oreg[i] = __float_as_uint(__uint_as_float(oreg[i]) * alpha);
+            tmem_st32(tO + c * 32, oreg);
+          }
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(P_FULL + x));
+      }
+      if (!ok) break;
+      // ---- epilogue: O / l -> bf16 -> shared -> global
+      ok = wait(O_FULL + x, n_o & 1u, 11);
+      if (!ok) break;
+      ++n_o;
+      tc_fence_after();
+      const float inv_l = 1.f / l;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t oreg[32];
+        tmem_ld32(tO + c * 32, oreg);
+        tmem_wait_ld();
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {      // four 16-byte chunks (8 bf16 each) per 32 columns
+          uint4 pk;
+          uint32_t* pw = reinterpret_cast<uint32_t*>(&pk);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(oreg[v * 8 + 2 * i]) * inv_l,
+                                                     __uint_as_float(oreg[v * 8 + 2 * i + 1]) * inv_l);
+            pw[i] = *reinterpret_cast<uint32_t*>(&t);
+          }
+          const int chunk = c * 4 + v;     // 16-byte chunk index inside the row
+          *reinterpret_cast<uint4*>(stage + r * (D * 2) + ((chunk ^ (r & 7)) * 16)) = pk;
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(bar(O_EMPTY + x));        // TMEM O (and S) of this tile may be overwritten
+      if (lse != nullptr && tile_row0 + r < it.hi)
+        lse[(size_t)it.bh * T + tile_row0 + r] = m * scale + __logf(l);
+      mbar_arrive(bar(STG_FULL + x));          // all 128 rows staged (bounded wait, no bar.sync)
+      ok = wait(STG_FULL + x, (n_o & 1u) ^ 1u, 12);
+      if (!ok) break;
+      constexpr int kChunks = D * 2 / 16;   // 16-byte chunks per row
+      const int t = threadIdx.x - (4 + 4 * x) * 32;
+#pragma unroll 4
+      for (int id = t; id < kTileM * kChunks; id += kTileM) {
+        const int row = id / kChunks, chunk = id % kChunks;
+        if (tile_row0 + row < it.hi) {
+          const uint4 val = *reinterpret_cast<const uint4*>(stage + row * (D * 2) + ((chunk ^ (row & 7)) * 16));
+          *reinterpret_cast<uint4*>(Op + ((size_t)it.bh * T + tile_row0 + row) * D + chunk * 8) = val;
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(bar(Q_EMPTY + x));        // the producer may load the next Q tile here
+    }
+  }
+
+  __syncwarp();
+  // ----------------------------------------------------------------------------- teardown
+  if (*abort_flag) {
+    // give copies and MMAs already in flight time to land before the TMEM is released
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+  }
+}
+
+// ----------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// [B*H, T, D] bf16, box 64 x 128 x 1, 128-byte swizzle, out-of-range rows read as zero.
+bool make_map(CUtensorMap* map, const void* ptr, int D, long long T, long long BH) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)T, (cuuint64_t)BH};
+  cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)T * D * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)kTileM, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D>
+moga_status launch(const moga_shape& s, const WsLayout& L, const void* Qp, const void* Kp, const void* Vp,
+                   const int32_t* offsets, void* Op, float* lse, char* ws, cudaStream_t st) {
+  const long long T = (long long)s.N * s.k;
+  CUtensorMap mq, mk, mv;
+  if (!make_map(&mq, Qp, D, T, (long long)s.B * s.H) || !make_map(&mk, Kp, D, T, (long long)s.B * s.H) ||
+      !make_map(&mv, Vp, D, T, (long long)s.B * s.H))
+    return MOGA_ERR_CUDA;
+  int32_t* order = reinterpret_cast<int32_t*>(ws + L.sched);
+  int32_t* prefix = order + (size_t)s.B * s.M;
+  uint32_t* header = reinterpret_cast<uint32_t*>(ws + L.header);
+  attn_schedule_kernel<<<1, 256, 0, st>>>(offsets, order, prefix, s.B, s.M, s.H);
+  MOGA_CUDA_OK(cudaGetLastError());
+  static int num_sms = 0;
+  if (num_sms == 0) {
+    int dev = 0;
+    MOGA_CUDA_OK(cudaGetDevice(&dev));
+    MOGA_CUDA_OK(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
+  }
+  auto kern = attn_bf16_kernel<D>;
+  MOGA_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::kDynSmem));
+  const long long max_items = ((T + kQBlock - 1) / kQBlock + s.M) * (long long)s.B * s.H;
+  const int grid = (int)(max_items < num_sms ? max_items : num_sms);
+  const float log2e = 1.4426950408889634f;
+  kern<<<grid, kThreads, Cfg<D>::kDynSmem, st>>>(mq, mk, mv, offsets, order, prefix,
+                                                  static_cast<__nv_bfloat16*>(Op), lse, header, (int)T, s.H,
+                                                  s.M, s.B * s.M, s.scale * log2e, s.scale);
+  MOGA_CUDA_OK(cudaGetLastError());
+  return MOGA_OK;
+}
+
+}  // namespace
+
+moga_status launch_attn_bf16(const moga_shape& s, const WsLayout& L, const void* Qp, const void* Kp,
+                             const void* Vp, const int32_t* offsets, void* Op, float* lse, char* ws,
+                             cudaStream_t st) {
+  if ((long long)s.N * s.k == 0) return MOGA_OK;
+  if (s.D == 128) return launch<128>(s, L, Qp, Kp, Vp, offsets, Op, lse, ws, st);
+  return launch<64>(s, L, Qp, Kp, Vp, offsets, Op, lse, ws, st);
+}
+
 }  // namespace moga

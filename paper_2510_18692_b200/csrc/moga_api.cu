@@ -13,7 +13,7 @@ bool check_shape(const moga_shape* s, moga_status* st) {
   if (s->B < 1 || s->N < 0 || s->H < 1 || s->C < 1 || s->D < 1 || s->M < 1 || s->k < 1 ||
       (s->dtype != MOGA_F32 && s->dtype != MOGA_BF16) ||
       (s->gate_mode != MOGA_GATE_SOFTMAX_ALL && s->gate_mode != MOGA_GATE_SOFTMAX_TOPK) ||
-      !(s->scale == s->scale)) {
+      !(s->scale >= 0.f) || s->scale > 3.0e38f) {
     *st = MOGA_ERR_INVALID_ARG;
     return false;
   }
