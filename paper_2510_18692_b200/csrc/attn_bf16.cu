@@ -447,9 +447,13 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
           for (int c = 0; c < 128; ++c)
             if (c >= ncols) sreg[c] = 0xff800000u;        // -inf
         }
-        float mt = __uint_as_float(sreg[0]);
+        float mx[8];
 #pragma unroll
-        for (int c = 1; c < 128; ++c) mt = fmaxf(mt, __uint_as_float(sreg[c]));
+        for (int c = 0; c < 8; ++c) mx[c] = __uint_as_float(sreg[c]);
+#pragma unroll
+        for (int c = 8; c < 128; ++c) mx[c & 7] = fmaxf(mx[c & 7], __uint_as_float(sreg[c]));
+        const float mt = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                               fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
         const float m_new = fmaxf(m, mt);
         // keep the old maximum unless it is stale by more than 2^8 somewhere in this warp
         const bool grow = j == 0 || (m_new - m) * scale_log2 > 8.0f;
@@ -460,16 +464,17 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
           m = m_new;
         }
         const float neg_m = -m * scale_log2;
-        float lsum = 0.f;
+        float ls[4] = {0.f, 0.f, 0.f, 0.f};
         uint32_t preg[64];
 #pragma unroll
         for (int c = 0; c < 64; ++c) {
           const float p0 = ex2(fmaf(__uint_as_float(sreg[2 * c]), scale_log2, neg_m));
           const float p1 = ex2(fmaf(__uint_as_float(sreg[2 * c + 1]), scale_log2, neg_m));
-          lsum += p0 + p1;
+          ls[c & 3] += p0 + p1;
           __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
           preg[c] = *reinterpret_cast<uint32_t*>(&pk);
         }
+        const float lsum = (ls[0] + ls[1]) + (ls[2] + ls[3]);
         l = l * alpha + lsum;
         tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&preg[0]));
         tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&preg[32]));
