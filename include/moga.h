@@ -99,6 +99,34 @@ moga_status moga_permute(const moga_shape* s, const int32_t* gid, const void* Q,
                          void* Kp, void* Vp, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Group sort without a caller workspace (the paper has no counterpart: this entry
+ * point exists for the way the library is hosted, not for the method).
+ *
+ * It computes exactly what moga_permute computes when Qp, Kp and Vp are NULL --
+ * perm, inv and offsets from gid -- but keeps its scratch (a 256-byte status header
+ * and B * ceil(N*k / 4096) * M int32 block counters) in a 1 MiB device array that is
+ * part of the library image, so the call performs no device allocation of any kind.
+ * It is meant for hosts that cannot allocate when they need the sort: code running
+ * inside another framework's execution step whose pool already owns the GPU's
+ * memory, or a service whose device-memory budget was fixed at start-up.
+ *
+ *  - Shapes whose counters do not fit the array return MOGA_ERR_WORKSPACE and launch
+ *    nothing (all of this library's documented workloads fit with room to spare).
+ *  - Every GPU that loads the library holds the 1 MiB until the process exits.
+ *  - The first call on each device looks the array's address up for that device;
+ *    make that first call outside any stream capture.
+ *  - All calls on a device share the array.  Each call clears the status header it
+ *    needs and overwrites the counters, so consecutive calls on one stream are
+ *    independent, but two calls that overlap on the GPU (different streams) race:
+ *    serialise them.
+ *  - status_out, if non-NULL, is a device pointer to two uint32 (8-byte aligned) that
+ *    receives {status, detail} as moga_last_device_status would report them, e.g.
+ *    MOGA_ERR_INTERNAL for a gid outside [0, M) (which is clamped).
+ */
+moga_status moga_sort_static(const moga_shape* s, const int32_t* gid, int32_t* perm, int32_t* inv,
+                             int32_t* offsets, uint32_t* status_out, void* stream);
+
+/*
  * Alg. 1 line 3 / Eq. 1 inside each group: for every (b, h, g),
  * Op_g = softmax(Qp_g Kp_g^T * scale) Vp_g, non-causal, no mask but the group
  * boundary.  bf16 runs on tcgen05 tensor cores (fp32 accumulate and softmax);

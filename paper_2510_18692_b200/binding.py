@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libmoga.so")
 
 EXPORTS = ("moga_workspace_bytes", "moga_scratch_bytes", "moga_status_string", "moga_route",
            "moga_permute", "moga_group_attn", "moga_unpermute", "moga_forward",
-           "moga_last_device_status")
+           "moga_last_device_status", "moga_sort_static")
 
 MOGA_F32, MOGA_BF16 = 0, 1
 STATUS_NAMES = {0: "MOGA_OK", 1: "MOGA_ERR_INVALID_ARG", 2: "MOGA_ERR_UNSUPPORTED",
@@ -99,6 +99,12 @@ def moga_permute(shape, gid, Q, K, V, perm, inv, offsets, Qp, Kp, Vp, ws):
     _check(lib.moga_permute(ctypes.byref(shape), _ptr(gid), _ptr(Q), _ptr(K), _ptr(V), _ptr(perm),
                             _ptr(inv), _ptr(offsets), _ptr(Qp), _ptr(Kp), _ptr(Vp), _ptr(ws),
                             ctypes.c_size_t(ws.numel()), _stream()), "moga_permute")
+
+
+def moga_sort_static(shape, gid, perm, inv, offsets, status_out=None):
+    """Group sort with library-resident scratch: no workspace, no device allocation."""
+    _check(lib.moga_sort_static(ctypes.byref(shape), _ptr(gid), _ptr(perm), _ptr(inv), _ptr(offsets),
+                                _ptr(status_out), _stream()), "moga_sort_static")
 
 
 def moga_group_attn(shape, Qp, Kp, Vp, offsets, Op, lse, ws):
