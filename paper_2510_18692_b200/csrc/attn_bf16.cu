@@ -80,20 +80,26 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                : "memory");
 }
+// Matrix descriptors are passed as (low word, high word): the high word is a constant of the
+// layout, the low word carries the start address, so stepping through a tile is a 32-bit add.
 // D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+__device__ __forceinline__ void mma_ss(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t ab_hi,
+                                       uint32_t idesc, uint32_t acc) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc)
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d), "r"(a_lo), "r"(b_lo), "r"(ab_hi), "r"(idesc), "r"(acc)
       : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                       uint32_t acc) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc)
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+      ::"r"(d), "r"(a), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(acc)
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -128,10 +134,20 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// Shared-memory matrix descriptor, 128-byte swizzle.  lbo/sbo in bytes.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
-  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
-         (1ull << 46) | (2ull << 61);
+template <int N>
+__device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle, split in two words.  Low word: start
+// address (bits 0-13, in 16-byte units) and leading byte offset (bits 16-29); high word:
+// stride byte offset (bits 0-13), descriptor version 1 (bit 14), layout type SWIZZLE_128B
+// (value 2 in bits 29-31).
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
+  return ((addr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
+}
+__host__ __device__ constexpr uint32_t desc_hi(uint32_t sbo_bytes) {
+  return (sbo_bytes >> 4) | (1u << 14) | (2u << 29);
 }
 // kind::f16 instruction descriptor: bf16 x bf16 -> f32, A K-major, B K-major or MN-major.
 __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major) {
@@ -294,6 +310,12 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     return true;
   };
 
+  // Registers move from the producer / MMA warpgroup (warps 0-3) to the softmax warpgroups:
+  // 128 * 80 + 256 * 208 <= 384 * 168.
+  // (each setmaxnreg sits at the top of the branch it governs, so the compiler can give
+  //  the code it dominates that many registers)
+  if (warp < 4) {
+    reg_dec<80>();
   if (warp == 0) {
     // ===================================================================== TMA producer
     if (lane == 0) {
@@ -342,22 +364,22 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       uint32_t nq[2] = {0, 0}, ns[2] = {0, 0}, np[2] = {0, 0}, no[2] = {0, 0}, nk = 0, nv = 0;
       bool ok = true;
       // S_x = Q_x K^T for the K tile in ring slot s
+      constexpr uint32_t hi = desc_hi(1024);   // 8-row groups are 1024 bytes apart in every tile
       auto issue_qk = [&](int x, int s) {
-        const uint32_t qa = sQ + x * C::kTileBytes, kb = sK + s * C::kTileBytes;
+        const uint32_t qa = desc_lo(sQ + x * C::kTileBytes, 16), kb = desc_lo(sK + s * C::kTileBytes, 16);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t o = (kk / 4) * C::kBoxBytes + (kk % 4) * 32;
-          mma_ss(tmem + x * kTileN, smem_desc(qa + o, 16, 1024), smem_desc(kb + o, 16, 1024), idesc_qk,
-                 kk > 0);
+          const uint32_t o = ((kk / 4) * C::kBoxBytes + (kk % 4) * 32) >> 4;
+          mma_ss(tmem + x * kTileN, qa + o, kb + o, hi, idesc_qk, kk > 0);
         }
       };
-      // O_x (+)= P_x V for the V tile in ring slot s
+      // O_x (+)= P_x V for the V tile in ring slot s (V is MN-major: 64-column boxes kBoxBytes apart)
       auto issue_pv = [&](int x, int s, bool accumulate) {
-        const uint32_t vb = sV + s * C::kTileBytes;
+        const uint32_t vb = desc_lo(sV + s * C::kTileBytes, C::kBoxBytes);
 #pragma unroll
         for (int kk = 0; kk < kTileN / 16; ++kk)
-          mma_ts(tmem + 256 + x * 128, tmem + x * kTileN + kk * 8,
-                 smem_desc(vb + kk * 2048, C::kBoxBytes, 1024), idesc_pv, (accumulate || kk > 0) ? 1u : 0u);
+          mma_ts(tmem + 256 + x * 128, tmem + x * kTileN + kk * 8, vb + ((kk * 2048) >> 4), hi, idesc_pv,
+                 (accumulate || kk > 0) ? 1u : 0u);
       };
       for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
         const Item it = decode_item(w, offsets, order, prefix, BM, M, H);
@@ -415,8 +437,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       }
       (void)ns;
     }
-  } else if (warp >= 4) {
+  }
+  } else {
     // ===================================================================== softmax + epilogue
+    reg_inc<208>();
     const int x = (warp - 4) >> 2;                 // 0: tile A, 1: tile B
     const int q = warp & 3;                        // TMEM lane quarter of this warp
     const int r = q * 32 + lane;                   // row inside the tile
@@ -464,17 +488,20 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
           m = m_new;
         }
         const float neg_m = -m * scale_log2;
-        float ls[4] = {0.f, 0.f, 0.f, 0.f};
+        const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(neg_m, neg_m);
+        float2 ls[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
         uint32_t preg[64];
 #pragma unroll
         for (int c = 0; c < 64; ++c) {
-          const float p0 = ex2(fmaf(__uint_as_float(sreg[2 * c]), scale_log2, neg_m));
-          const float p1 = ex2(fmaf(__uint_as_float(sreg[2 * c + 1]), scale_log2, neg_m));
-          ls[c & 3] += p0 + p1;
-          __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+          const float2 x = __ffma2_rn(make_float2(__uint_as_float(sreg[2 * c]), __uint_as_float(sreg[2 * c + 1])),
+                                      sc2, nm2);
+          const float2 pe = make_float2(ex2(x.x), ex2(x.y));
+          ls[c & 3] = __fadd2_rn(ls[c & 3], pe);
+          __nv_bfloat162 pk = __floats2bfloat162_rn(pe.x, pe.y);
           preg[c] = *reinterpret_cast<uint32_t*>(&pk);
         }
-        const float lsum = (ls[0] + ls[1]) + (ls[2] + ls[3]);
+        const float2 l01 = __fadd2_rn(__fadd2_rn(ls[0], ls[1]), __fadd2_rn(ls[2], ls[3]));
+        const float lsum = l01.x + l01.y;
         l = l * alpha + lsum;
         tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&preg[0]));
         tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&preg[32]));
