@@ -10,9 +10,10 @@
 //   warp 1      MMA issuer (one lane): S = Q K^T into TMEM, O += P V with P read
 //               from TMEM; owns the TMEM allocation.
 //   warps 4-7   softmax of tile A, one thread per query row; warps 8-11 tile B.
-//               Online softmax in the log2 domain with a lazily updated maximum:
-//               O is rescaled (in TMEM, by the same warps) only when the row
-//               maximum grew by more than 2^8.  They also run the epilogue:
+//               Online softmax in the log2 domain against a reference maximum taken
+//               from the row's first tile; it is raised, and O rescaled in TMEM by
+//               the same warps, only when a later tile's row sum exceeds 2^40.
+//               They also run the epilogue:
 //               O / l -> bf16 -> shared memory -> coalesced, row-predicated stores.
 //
 // TMEM (512 columns): S_A [0,128) S_B [128,256) O_A [256,256+D) O_B [384,384+D);
@@ -31,6 +32,7 @@ constexpr int kTileM = 128;       // query rows per tile
 constexpr int kTileN = 128;       // keys per K/V tile
 constexpr int kQBlock = 2 * kTileM;
 constexpr uint64_t kWaitLimitNs = 4000000000ull;  // 4 s: far above any legitimate wait
+constexpr float kRowSumLimit = 1.0995116e12f;      // 2^40: a tile's row sum beyond this forces a new maximum
 
 // ----------------------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -461,47 +463,55 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         if (!ok) break;
         ++n_s;
         tc_fence_after();
-        uint32_t sreg[128];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
-        tmem_wait_ld();
-        const int ncols = it.hi - it.lo - j * kTileN;     // valid keys in this tile (may exceed 128)
-        if (ncols < kTileN) {
-#pragma unroll
-          for (int c = 0; c < 128; ++c)
-            if (c >= ncols) sreg[c] = 0xff800000u;        // -inf
-        }
-        float mx[8];
-#pragma unroll
-        for (int c = 0; c < 8; ++c) mx[c] = __uint_as_float(sreg[c]);
-#pragma unroll
-        for (int c = 8; c < 128; ++c) mx[c & 7] = fmaxf(mx[c & 7], __uint_as_float(sreg[c]));
-        const float mt = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
-                               fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
-        const float m_new = fmaxf(m, mt);
-        // keep the old maximum unless it is stale by more than 2^8 somewhere in this warp
-        const bool grow = j == 0 || (m_new - m) * scale_log2 > 8.0f;
-        const bool rescale = __any_sync(0xffffffffu, grow);
-        float alpha = 1.f;
-        if (rescale) {
-          alpha = j == 0 ? 0.f : ex2((m - m_new) * scale_log2);
-          m = m_new;
-        }
-        const float neg_m = -m * scale_log2;
-        const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(neg_m, neg_m);
-        float2 ls[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+        // Tile 0 fixes the row's reference maximum m.  Later tiles exponentiate against the
+        // same m without looking for their own maximum: any reference gives the same quotient
+        // O / l as long as nothing overflows, and bf16 / fp32 keep their relative precision at
+        // any magnitude.  Only when a row sum shows scores far above m (2^40, inf or nan) is the
+        // tile redone with its exact maximum, m raised, and O and l rescaled.
         uint32_t preg[64];
+        float alpha = 1.f, lsum;
+        bool exact = (j == 0), rescale = false;
+        const int ncols = it.hi - it.lo - j * kTileN;     // valid keys in this tile (may exceed 128)
+        while (true) {
+          uint32_t sreg[128];
 #pragma unroll
-        for (int c = 0; c < 64; ++c) {
-          const float2 x = __ffma2_rn(make_float2(__uint_as_float(sreg[2 * c]), __uint_as_float(sreg[2 * c + 1])),
-                                      sc2, nm2);
-          const float2 pe = make_float2(ex2(x.x), ex2(x.y));
-          ls[c & 3] = __fadd2_rn(ls[c & 3], pe);
-          __nv_bfloat162 pk = __floats2bfloat162_rn(pe.x, pe.y);
-          preg[c] = *reinterpret_cast<uint32_t*>(&pk);
+          for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
+          tmem_wait_ld();
+          if (ncols < kTileN) {
+#pragma unroll
+            for (int c = 0; c < 128; ++c)
+              if (c >= ncols) sreg[c] = 0xff800000u;        // -inf
+          }
+          if (exact) {
+            float mx[8];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) mx[c] = __uint_as_float(sreg[c]);
+#pragma unroll
+            for (int c = 8; c < 128; ++c) mx[c & 7] = fmaxf(mx[c & 7], __uint_as_float(sreg[c]));
+            const float mt = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                                   fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+            const float m_new = fmaxf(m, mt);
+            alpha = j == 0 ? 0.f : ex2((m - m_new) * scale_log2);
+            m = m_new;
+            rescale = j > 0;
+          }
+          const float neg_m = -m * scale_log2;
+          const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(neg_m, neg_m);
+          float2 ls[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+#pragma unroll
+          for (int c = 0; c < 64; ++c) {
+            const float2 x = __ffma2_rn(make_float2(__uint_as_float(sreg[2 * c]), __uint_as_float(sreg[2 * c + 1])),
+                                        sc2, nm2);
+            const float2 pe = make_float2(ex2(x.x), ex2(x.y));
+            ls[c & 3] = __fadd2_rn(ls[c & 3], pe);
+            __nv_bfloat162 pk = __floats2bfloat162_rn(pe.x, pe.y);
+            preg[c] = *reinterpret_cast<uint32_t*>(&pk);
+          }
+          const float2 l01 = __fadd2_rn(__fadd2_rn(ls[0], ls[1]), __fadd2_rn(ls[2], ls[3]));
+          lsum = l01.x + l01.y;
+          if (exact || !__any_sync(0xffffffffu, !(lsum < kRowSumLimit))) break;
+          exact = true;       // S is still intact in TMEM: load it again and take the maximum
         }
-        const float2 l01 = __fadd2_rn(__fadd2_rn(ls[0], ls[1]), __fadd2_rn(ls[2], ls[3]));
-        const float lsum = l01.x + l01.y;
         l = l * alpha + lsum;
         tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&preg[0]));
         tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&preg[32]));

@@ -231,3 +231,38 @@ def test_group_attn_peaky_bf16(mb):
     check_output(Op.float().cpu().numpy(), want, "bf16", "Op")
     rel = np.linalg.norm(Op.float().cpu().numpy() - want) / np.linalg.norm(want)
     assert rel < 2e-2
+
+
+@pytest.mark.parametrize("grow", [3.0, 24.0])
+def test_group_attn_growing_scores_bf16(mb, grow):
+    """Keys late in each group are scaled up, so later K/V tiles hold scores far above the
+    first tile's maximum: x3 stays on the kernel's fixed-reference path with large positive
+    exponents, x24 overflows it and forces the mid-row change of reference.  Outputs are
+    O(1) here (a few keys dominate each row), so the bound is relative."""
+    sizes = [900, 515, 130]
+    case = grouped_case(sizes, 2, 128, "bf16", seed=11, B=1)
+    off = case["offsets"][0]
+    for g in range(len(sizes)):
+        lo, hi = int(off[g]), int(off[g + 1])
+        case["K"][:, :, lo + (hi - lo) // 3:hi] *= grow
+    cfg = _cfg(B=1, H=2, N=case["T"], D=128, M=len(sizes), k=1, dtype="bf16")
+    scale = 1.0 / math.sqrt(128)
+    sh = mb.make_shape(cfg, scale=scale)
+    Op = torch.full_like(case["Q"], float("nan"))
+    lse = torch.empty(1, 2, case["T"], dtype=torch.float32, device="cuda")
+    ws = mb.alloc_workspace(mb.moga_scratch_bytes(sh))
+    mb.moga_group_attn(sh, case["Q"], case["K"], case["V"], torch.from_numpy(case["offsets"]).cuda(), Op,
+                       lse, ws)
+    assert mb.moga_last_device_status(ws) == (0, 0)
+    want = oracle.attn_all(to_np32(case["Q"]), to_np32(case["K"]), to_np32(case["V"]), case["gid"],
+                           np.ones((1, case["T"], 1)), case["offsets"], case["perm"], scale)
+    got = Op.float().cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(got))
+    assert np.linalg.norm(got - want) / np.linalg.norm(want) < 1e-2
+    assert np.abs(got - want).max() <= 2.0 ** -6 * np.abs(want).max()
+    q, k_ = case["Q"].double().cpu(), case["K"].double().cpu()
+    for g in range(len(sizes)):
+        lo, hi = int(off[g]), int(off[g + 1])
+        s = torch.einsum("bhnd,bhmd->bhnm", q[:, :, lo:hi], k_[:, :, lo:hi]) * scale
+        ref = torch.logsumexp(s, -1)
+        assert (lse[:, :, lo:hi].double().cpu() - ref).abs().max().item() <= 2e-2
