@@ -35,7 +35,7 @@ from paper_2510_18692_b200.inputs import CONFIGS, make_inputs, useful_flops  # n
 
 METRIC = "MoGA fwd effective TFLOP/s (bf16)"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-KERNELS_PER_FORWARD = 8   # route, 3 sort kernels, gather, attention schedule, attention, unpermute
+KERNELS_PER_FORWARD = 9   # weight split, route, 3 sort kernels, gather, attention schedule, attention, unpermute
 
 
 def load_peaks():
@@ -257,7 +257,7 @@ def main():
     for it in range(args.steps + 1):
         e = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
         e[0].record()
-        mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], gid, gate, None)
+        mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], gid, gate, None, ws)
         e[1].record()
         mb.moga_permute(sh, gid, inp["Q"], inp["K"], inp["V"], perm, inv, offsets, Qp, Kp, Vp, ws)
         e[2].record()

@@ -61,12 +61,20 @@ typedef enum {
   MOGA_GATE_SOFTMAX_TOPK = 1 /* gate = softmax over the k selected logits               */
 } moga_gate_mode;
 
+typedef enum {
+  MOGA_ROUTE_AUTO = 0, /* bf16 X and a workspace: tensor-core router (fp32 weights as three
+                          bf16 parts, exact products, fp32 accumulation); otherwise fp32 ALUs */
+  MOGA_ROUTE_ALU = 1   /* always the fp32-ALU router kernel                                 */
+} moga_route_mode;
+
 typedef struct {
   int32_t B, N, H, C, D, M, k;
   int32_t dtype;     /* moga_dtype of X, Q, K, V, O and the permuted buffers            */
   int32_t gate_mode; /* moga_gate_mode                                                  */
   float scale;       /* softmax scale of Eq. 1, e.g. 1/sqrt(D); finite, >= 0; never inferred */
   int64_t q_stride_b, q_stride_h, q_stride_n; /* element strides of Q, K, V and O       */
+  int32_t route_mode; /* moga_route_mode                                                 */
+  int32_t reserved;   /* set to 0                                                        */
 } moga_shape;
 
 /* Host-only helpers: no CUDA call is made. */
@@ -80,7 +88,13 @@ const char* moga_status_string(moga_status st);
 /*
  * Router, Eq. 2-4: r = X W_r (+ bias) accumulated in fp32, the k largest logits
  * per token (ties to the lower group index), and their gates (gate_mode).
- * Writes gid, gate and, if non-NULL, logits.  Needs no workspace (ws may be NULL).
+ * Writes gid, gate and, if non-NULL, logits.
+ * Two kernels compute the same thing to fp32 rounding.  The fp32-ALU kernel needs no
+ * workspace (ws may be NULL) and serves fp32 X.  For bf16 X, when ws holds at least
+ * moga_scratch_bytes and route_mode is MOGA_ROUTE_AUTO, the tensor-core kernel runs: it
+ * writes each fp32 weight as the sum of three bf16 numbers (all 24 mantissa bits), so
+ * every product with a bf16 feature is exact, and accumulates in fp32.  That call resets
+ * and may set the device status word of ws (see moga_last_device_status).
  */
 moga_status moga_route(const moga_shape* s, const void* X, const float* Wr, const float* bias,
                        int32_t* gid, float* gate, float* logits, void* ws, size_t ws_bytes,

@@ -22,6 +22,7 @@ EXPORTS = ("moga_workspace_bytes", "moga_scratch_bytes", "moga_status_string", "
            "moga_last_device_status", "moga_sort_static")
 
 MOGA_F32, MOGA_BF16 = 0, 1
+MOGA_ROUTE_AUTO, MOGA_ROUTE_ALU = 0, 1
 STATUS_NAMES = {0: "MOGA_OK", 1: "MOGA_ERR_INVALID_ARG", 2: "MOGA_ERR_UNSUPPORTED",
                 3: "MOGA_ERR_WORKSPACE", 4: "MOGA_ERR_CUDA", 5: "MOGA_ERR_TIMEOUT",
                 6: "MOGA_ERR_INTERNAL"}
@@ -32,7 +33,8 @@ class MogaShape(ctypes.Structure):
                 ("C", ctypes.c_int32), ("D", ctypes.c_int32), ("M", ctypes.c_int32),
                 ("k", ctypes.c_int32), ("dtype", ctypes.c_int32), ("gate_mode", ctypes.c_int32),
                 ("scale", ctypes.c_float), ("q_stride_b", ctypes.c_int64),
-                ("q_stride_h", ctypes.c_int64), ("q_stride_n", ctypes.c_int64)]
+                ("q_stride_h", ctypes.c_int64), ("q_stride_n", ctypes.c_int64),
+                ("route_mode", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 class MogaError(RuntimeError):
@@ -56,11 +58,11 @@ def status_string(code: int) -> str:
     return lib.moga_status_string(ctypes.c_int(code)).decode()
 
 
-def make_shape(cfg: MogaConfig, strides=None, scale=None) -> MogaShape:
+def make_shape(cfg: MogaConfig, strides=None, scale=None, route_mode=MOGA_ROUTE_AUTO) -> MogaShape:
     sb, sh, sn = strides if strides is not None else (0, 0, 0)
     return MogaShape(cfg.B, cfg.N, cfg.H, cfg.C, cfg.D, cfg.M, cfg.k,
                      MOGA_F32 if cfg.dtype == "f32" else MOGA_BF16, cfg.gate_mode,
-                     cfg.scale if scale is None else scale, sb, sh, sn)
+                     cfg.scale if scale is None else scale, sb, sh, sn, route_mode, 0)
 
 
 def _ptr(t):

@@ -13,6 +13,7 @@ bool check_shape(const moga_shape* s, moga_status* st) {
   if (s->B < 1 || s->N < 0 || s->H < 1 || s->C < 1 || s->D < 1 || s->M < 1 || s->k < 1 ||
       (s->dtype != MOGA_F32 && s->dtype != MOGA_BF16) ||
       (s->gate_mode != MOGA_GATE_SOFTMAX_ALL && s->gate_mode != MOGA_GATE_SOFTMAX_TOPK) ||
+      (s->route_mode != MOGA_ROUTE_AUTO && s->route_mode != MOGA_ROUTE_ALU) ||
       !(s->scale >= 0.f) || s->scale > 3.0e38f) {
     *st = MOGA_ERR_INVALID_ARG;
     return false;
@@ -51,6 +52,13 @@ moga_status clear_header(char* ws, const WsLayout& L, cudaStream_t st) {
 
 #define PTR_OK(p) ((p) != nullptr && aligned16(p))
 
+// bf16 features go to the tensor-core router when the caller provides scratch for the split
+// weights and has not asked for the fp32-ALU kernel; everything else runs on the fp32 ALUs.
+bool route_on_tensor_cores(const moga_shape& s, const WsLayout& L, const void* ws, size_t ws_bytes) {
+  return s.dtype == MOGA_BF16 && s.route_mode == MOGA_ROUTE_AUTO && ws != nullptr &&
+         ws_bytes >= L.scratch_end && (reinterpret_cast<uintptr_t>(ws) & (kWsAlign - 1)) == 0;
+}
+
 }  // namespace
 
 extern "C" {
@@ -83,14 +91,19 @@ const char* moga_status_string(moga_status st) {
 moga_status moga_route(const moga_shape* s, const void* X, const float* Wr, const float* bias,
                        int32_t* gid, float* gate, float* logits, void* ws, size_t ws_bytes,
                        void* stream) {
-  (void)ws;
-  (void)ws_bytes;
   moga_status st;
   if (!check_shape(s, &st)) return st;
   if (!PTR_OK(X) || !PTR_OK(Wr) || !PTR_OK(gid) || !PTR_OK(gate) ||
       (bias != nullptr && !aligned16(bias)) || (logits != nullptr && !aligned16(logits)))
     return MOGA_ERR_INVALID_ARG;
-  return launch_route(*s, X, Wr, bias, gid, gate, logits, static_cast<cudaStream_t>(stream));
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const WsLayout L = ws_layout(*s);
+  if (route_on_tensor_cores(*s, L, ws, ws_bytes)) {
+    char* w = static_cast<char*>(ws);
+    if ((st = clear_header(w, L, cs)) != MOGA_OK) return st;
+    return launch_route_mma(*s, L, X, Wr, bias, gid, gate, logits, w, cs);
+  }
+  return launch_route(*s, X, Wr, bias, gid, gate, logits, cs);
 }
 
 moga_status moga_permute(const moga_shape* s, const int32_t* gid, const void* Q, const void* K,
@@ -164,7 +177,10 @@ moga_status moga_forward(const moga_shape* s, const void* X, const float* Wr, co
   void* Vp = w + L.Vp;
   void* Op = w + L.Op;
   if ((st = clear_header(w, L, cs)) != MOGA_OK) return st;
-  if ((st = launch_route(*s, X, Wr, bias, gid, gate, nullptr, cs)) != MOGA_OK) return st;
+  st = route_on_tensor_cores(*s, L, ws, ws_bytes)
+           ? launch_route_mma(*s, L, X, Wr, bias, gid, gate, nullptr, w, cs)
+           : launch_route(*s, X, Wr, bias, gid, gate, nullptr, cs);
+  if (st != MOGA_OK) return st;
   if ((st = launch_sort(*s, L, gid, perm, inv, offsets, w, cs)) != MOGA_OK) return st;
   if ((st = launch_gather(*s, perm, Q, K, V, Qp, Kp, Vp, cs)) != MOGA_OK) return st;
   if (s->dtype == MOGA_F32)

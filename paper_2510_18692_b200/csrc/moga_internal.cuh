@@ -25,6 +25,7 @@ struct WsLayout {
   size_t header;      // 256 B
   size_t sort_hist;   // int32 [B, nblk, M]   per-block histograms, then bases
   size_t sched;       // int32 [B, 3, M+1]    attention schedule (order, tile prefix, ...)
+  size_t wsplit;      // bf16 [3, MP, C]      router weight split into three bf16 parts (MP <= 64)
   size_t scratch_end; // == moga_scratch_bytes
   size_t gid, gate, perm, inv, offsets;  // routing results
   size_t Qp, Kp, Vp, Op;                 // permuted tensors
@@ -44,6 +45,7 @@ inline WsLayout ws_layout(const moga_shape& s) {
   L.header = off;      off = align_up(off + 256, kWsAlign);
   L.sort_hist = off;   off = align_up(off + sizeof(int32_t) * (size_t)s.B * L.nblk * s.M, kWsAlign);
   L.sched = off;       off = align_up(off + sizeof(int32_t) * (size_t)s.B * 4 * (s.M + 1) + 64, kWsAlign);
+  L.wsplit = off;      off = align_up(off + sizeof(uint16_t) * 3 * (size_t)kMaxM * s.C, kWsAlign);
   L.scratch_end = off;
   L.gid = off;         off = align_up(off + sizeof(int32_t) * (size_t)s.B * T, kWsAlign);
   L.gate = off;        off = align_up(off + sizeof(float) * (size_t)s.B * T, kWsAlign);
@@ -74,6 +76,9 @@ __device__ __forceinline__ void report_status(uint32_t* header, uint32_t code, u
 // Stage launchers (each returns MOGA_OK or MOGA_ERR_CUDA; arguments already validated).
 moga_status launch_route(const moga_shape& s, const void* X, const float* Wr, const float* bias,
                          int32_t* gid, float* gate, float* logits, cudaStream_t st);
+moga_status launch_route_mma(const moga_shape& s, const WsLayout& L, const void* X, const float* Wr,
+                             const float* bias, int32_t* gid, float* gate, float* logits, char* ws,
+                             cudaStream_t st);
 moga_status launch_sort(const moga_shape& s, const WsLayout& L, const int32_t* gid, int32_t* perm,
                         int32_t* inv, int32_t* offsets, char* ws, cudaStream_t st);
 moga_status launch_gather(const moga_shape& s, const int32_t* perm, const void* Q, const void* K,

@@ -7,6 +7,7 @@
 // token-per-thread top-k / gate epilogue, so nothing but gid, gate (and optionally
 // the logits) is written.
 #include "moga_internal.cuh"
+#include "route_select.cuh"
 
 namespace moga {
 namespace {
@@ -162,40 +163,7 @@ route_kernel(const XT* __restrict__ X, const float* __restrict__ Wr, const float
   for (int r = tid; r < TT; r += kRouteThreads) {
     const long long tok = tok0 + r;
     if (tok >= total_tokens) continue;
-    const float* row = ls + r * LP;
-    unsigned long long taken = 0ull;
-    float top = 0.f, zsel = 0.f;
-    float val[kMaxK];
-    int sel[kMaxK];
-#pragma unroll
-    for (int j = 0; j < kMaxK; ++j) {
-      if (j < k) {
-        int best = -1;
-        float bv = 0.f;
-        for (int i = 0; i < M; ++i) {
-          if ((taken >> i) & 1ull) continue;
-          float v = row[i];
-          if (best < 0 || v > bv) { best = i; bv = v; }   // strict >: ties keep the lower index
-        }
-        taken |= 1ull << best;
-        sel[j] = best;
-        val[j] = bv;
-        if (j == 0) top = bv;
-        zsel += expf(bv - top);
-      }
-    }
-    float Z = zsel;
-    if (gate_mode == MOGA_GATE_SOFTMAX_ALL) {
-      Z = 0.f;
-      for (int i = 0; i < M; ++i) Z += expf(row[i] - top);
-    }
-#pragma unroll
-    for (int j = 0; j < kMaxK; ++j) {
-      if (j < k) {
-        gid[tok * k + j] = sel[j];
-        gate[tok * k + j] = expf(val[j] - top) / Z;
-      }
-    }
+    select_and_gate(ls + r * LP, M, k, gate_mode, gid + tok * k, gate + tok * k);
   }
 }
 

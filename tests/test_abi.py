@@ -68,6 +68,8 @@ def test_bad_arguments_return_codes_without_launch(binding):
     for kw in (dict(B=0), dict(N=-1), dict(gate_mode=7)):
         bad = binding.make_shape(cfg.with_(**kw))
         assert lib.moga_route(ctypes.byref(bad), _fake(), _fake(), null, _fake(), _fake(), null, null, z, null) == 1
+    bad = binding.make_shape(cfg, route_mode=5)
+    assert lib.moga_route(ctypes.byref(bad), _fake(), _fake(), null, _fake(), _fake(), null, null, z, null) == 1
     # workspace missing or too small: nothing is launched
     need = binding.moga_workspace_bytes(sh)
     args = [ctypes.byref(sh)] + [_fake()] * 2 + [null] + [_fake()] * 4 + [null] * 4

@@ -40,17 +40,28 @@ ROUTE_CASES = [
     _cfg(dtype="bf16", M=64, k=2, gate_mode=GATE_SOFTMAX_TOPK, C=768, N=2051, zipf_bias=2.0, seed=4),
     _cfg(dtype="bf16", M=5, k=3, gate_mode=GATE_SOFTMAX_ALL, C=264, N=515, seed=5),
     _cfg(dtype="f32", M=33, k=8, gate_mode=GATE_SOFTMAX_TOPK, C=100, N=300, seed=6),
+    _cfg(dtype="bf16", M=32, C=5120, N=20000, seed=7),                 # long accumulation, many tiles per CTA
+    _cfg(dtype="bf16", M=3, k=2, gate_mode=GATE_SOFTMAX_TOPK, C=40, N=130, seed=8),   # less than one chunk
+    _cfg(dtype="bf16", M=64, k=8, gate_mode=GATE_SOFTMAX_ALL, C=2048, N=1, seed=9),   # a single token
 ]
 
 
+@pytest.mark.parametrize("path", ["alu", "tensor"])
 @pytest.mark.parametrize("cfg", ROUTE_CASES, ids=lambda c: f"{c.dtype}-M{c.M}-k{c.k}-C{c.C}-N{c.N}")
-def test_route(mb, cfg):
+def test_route(mb, cfg, path):
+    """Both router kernels against the fp64 oracle: the fp32-ALU kernel (no workspace) and,
+    for bf16 features, the tensor-core kernel (split weights, chosen when a workspace is given)."""
+    if path == "tensor" and cfg.dtype != "bf16":
+        pytest.skip("the tensor-core router takes bf16 features")
     inp = make_inputs(cfg, device="cuda", heads=[])
     sh = mb.make_shape(cfg)
+    ws = mb.alloc_workspace(mb.moga_scratch_bytes(sh)) if path == "tensor" else None
     gid = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.int32, device="cuda")
     gate = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.float32, device="cuda")
     logits = torch.empty(cfg.B, cfg.N, cfg.M, dtype=torch.float32, device="cuda")
-    mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], gid, gate, logits)
+    mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], gid, gate, logits, ws)
+    if ws is not None:
+        assert mb.moga_last_device_status(ws) == (0, 0)
     torch.cuda.synchronize()
     o_gid, o_gate, o_logits = oracle.route(to_np32(inp["X"]), to_np32(inp["Wr"]), to_np32(inp["bias"]),
                                            cfg.k, cfg.gate_mode, want_logits=True)
@@ -59,9 +70,18 @@ def test_route(mb, cfg):
     assert flips <= max(2, int(cfg.B * cfg.N * cfg.k * 1e-3))
     # without the optional logits output the decisions are the same bits
     gid2, gate2 = torch.empty_like(gid), torch.empty_like(gate)
-    mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], gid2, gate2, None)
+    mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], gid2, gate2, None, ws)
     torch.cuda.synchronize()
     assert torch.equal(gid, gid2) and torch.equal(gate, gate2)
+    if path == "tensor":
+        # route_mode = ALU overrides the choice even with a workspace: same bits as the ALU kernel alone
+        sh_alu = mb.make_shape(cfg, route_mode=mb.MOGA_ROUTE_ALU)
+        g3, g4 = torch.empty_like(gid), torch.empty_like(gid)
+        t3, t4 = torch.empty_like(gate), torch.empty_like(gate)
+        mb.moga_route(sh_alu, inp["X"], inp["Wr"], inp["bias"], g3, t3, None, ws)
+        mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], g4, t4, None, None)
+        torch.cuda.synchronize()
+        assert torch.equal(g3, g4) and torch.equal(t3, t4)
 
 
 def _random_gid(B, N, M, k, seed, skew=False, empty=()):
