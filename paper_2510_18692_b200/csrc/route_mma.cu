@@ -4,18 +4,20 @@
 // the M multiply-adds per loaded element are cheap.  Each fp32 weight is written as the sum
 // of three bf16 numbers (w = hi + mid + lo, 24 mantissa bits in all), so every product
 // x * w_part is a bf16 x bf16 product, exact in fp32, and the sums are accumulated in fp32
-// in TMEM: the result agrees with an fp32 FMA chain to fp32 rounding.  To keep the
-// accumulation error of the tensor core (one rounding per 16-channel step) below that of
-// such a chain, consecutive 64-channel chunks rotate over NACC independent accumulators,
-// which the epilogue adds in fp32.
+// in TMEM: the result agrees with an fp32 FMA chain to fp32 rounding.  The three parts are
+// stacked along the MMA's N dimension (one instruction per 16-channel step covers all of
+// them: the cost of a step is set by streaming the 128-token A operand, not by N), so each
+// part has its own accumulator columns.  To keep the accumulation error of the tensor core
+// (one rounding per step) near that of an fp32 chain, consecutive 64-channel chunks rotate
+// over NACC independent accumulators; the epilogue adds parts and accumulators in fp32.
 //
 //   prep kernel  splits W_r [C, M] fp32 into Wsplit [3, MP, C] bf16 (K-major rows, MP = M
 //                rounded up to 16 / 32 / 64, padding rows zero).
 //   main kernel  persistent, one CTA per SM, 128 tokens per tile:
 //     warp 0     TMA producer: per chunk one X box [128 tokens x 64 ch] and one Wsplit box
 //                [3*MP rows x 64 ch] into a ring of stages (128-byte swizzle).
-//     warp 1     MMA issuer: per chunk 4 k-steps x 3 weight parts of
-//                tcgen05.mma 128 x MP x 16 into accumulator (chunk mod NACC).
+//     warp 1     MMA issuer: per chunk 4 k-steps of tcgen05.mma 128 x (3*MP) x 16 into
+//                accumulator (chunk mod NACC).
 //     warps 2-5  epilogue, one thread per token: adds the accumulators, bias, then the
 //                top-k / gate selection shared with the fp32-ALU router kernel.
 // Every mbarrier wait is bounded; on expiry the CTA records MOGA_ERR_TIMEOUT and leaves.
@@ -36,8 +38,9 @@ constexpr uint64_t kWaitLimitNs = 4000000000ull;
 
 template <int MP>
 struct RCfg {
-  static constexpr int NACC = (512 / MP) < 16 ? (512 / MP) : 16;
-  static constexpr int kTmemCols = NACC * MP;              // 256 (MP = 16) or 512
+  static constexpr int NACC = 512 / (3 * MP);              // 10, 5, 2 for MP = 16, 32, 64
+  static constexpr int kAccCols = 3 * MP;                  // hi | mid | lo partial sums
+  static constexpr int kTmemCols = 512;
   static constexpr int kWBytes = 3 * MP * 128;
   static constexpr int kStageBytes = kXBytes + kWBytes;    // a multiple of 1024
   static constexpr int kLogitPitch = MP + 1;
@@ -146,7 +149,7 @@ route_mma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
   } else if (warp == 1) {
     // ===================================================================== MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc(kTok, MP, false);
+      constexpr uint32_t idesc = instr_desc(kTok, 3 * MP, false);
       constexpr uint32_t hi = desc_hi(1024);
       uint32_t n = 0, nt = 0;
       bool ok = true;
@@ -161,13 +164,10 @@ route_mma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
           tc_fence_after();
           const uint32_t xa = desc_lo(base + s * R::kStageBytes, 16);
           const uint32_t wb = desc_lo(base + s * R::kStageBytes + kXBytes, 16);
-          const uint32_t d = tmem + (uint32_t)((q % NACC) * MP);
+          const uint32_t d = tmem + (uint32_t)((q % NACC) * R::kAccCols);
 #pragma unroll
           for (int kk = 0; kk < kChunk / 16; ++kk)
-#pragma unroll
-            for (int t = 0; t < 3; ++t)
-              mma_ss(d, xa + kk * 2, wb + ((t * MP * 128) >> 4) + kk * 2, hi, idesc,
-                     (q >= NACC || kk > 0 || t > 0) ? 1u : 0u);
+            mma_ss(d, xa + kk * 2, wb + kk * 2, hi, idesc, (q >= NACC || kk > 0) ? 1u : 0u);
           tc_commit(bar(EMPTY + s));
         }
         if (ok) tc_commit(bar(ACC_FULL));
@@ -179,7 +179,7 @@ route_mma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
     const int row = q4 * 32 + lane;
     const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16);
     const int et = threadIdx.x - 64;                // 0..127 among the epilogue threads
-    const int valid_cols = (nch < NACC ? nch : NACC) * MP;
+    const int valid_cols = (nch < NACC ? nch : NACC) * R::kAccCols;
     uint32_t nt = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x, ++nt) {

@@ -43,6 +43,8 @@ ROUTE_CASES = [
     _cfg(dtype="bf16", M=32, C=5120, N=20000, seed=7),                 # long accumulation, many tiles per CTA
     _cfg(dtype="bf16", M=3, k=2, gate_mode=GATE_SOFTMAX_TOPK, C=40, N=130, seed=8),   # less than one chunk
     _cfg(dtype="bf16", M=64, k=8, gate_mode=GATE_SOFTMAX_ALL, C=2048, N=1, seed=9),   # a single token
+    _cfg(dtype="bf16", M=64, k=2, gate_mode=GATE_SOFTMAX_TOPK, C=5120, N=9000, seed=10),
+    _cfg(dtype="bf16", M=16, k=2, gate_mode=GATE_SOFTMAX_TOPK, C=5120, N=9000, seed=11),
 ]
 
 
