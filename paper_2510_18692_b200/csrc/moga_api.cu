@@ -186,10 +186,13 @@ moga_status moga_forward(const moga_shape* s, const void* X, const float* Wr, co
   if (s->dtype == MOGA_F32)
     st = launch_attn_f32(*s, static_cast<const float*>(Qp), static_cast<const float*>(Kp),
                          static_cast<const float*>(Vp), offsets, static_cast<float*>(Op), nullptr, cs);
+  else if (s->k == 1)   // one assignment per token: the attention epilogue is the gated scatter
+    st = launch_attn_bf16_scatter(*s, L, Qp, Kp, Vp, offsets, perm, gate, O, w, cs);
   else
     st = launch_attn_bf16(*s, L, Qp, Kp, Vp, offsets, Op, nullptr, w, cs);
   if (st != MOGA_OK) return st;
-  if ((st = launch_unpermute(*s, Op, inv, gate, O, cs)) != MOGA_OK) return st;
+  if (s->dtype == MOGA_F32 || s->k > 1)
+    if ((st = launch_unpermute(*s, Op, inv, gate, O, cs)) != MOGA_OK) return st;
   const size_t T = (size_t)s->N * s->k;
   if (gid_out) MOGA_CUDA_OK(cudaMemcpyAsync(gid_out, gid, sizeof(int32_t) * s->B * T, cudaMemcpyDeviceToDevice, cs));
   if (gate_out) MOGA_CUDA_OK(cudaMemcpyAsync(gate_out, gate, sizeof(float) * s->B * T, cudaMemcpyDeviceToDevice, cs));

@@ -91,6 +91,12 @@ moga_status launch_attn_bf16(const moga_shape& s, const WsLayout& L, const void*
                              const void* Vp, const int32_t* offsets, void* Op, float* lse, char* ws,
                              cudaStream_t st);
 
+// Top-1 routing only: the attention epilogue writes gate * row straight to token order in O
+// (the gated inverse permutation of Eq. 5), so no permuted output and no unpermute pass.
+moga_status launch_attn_bf16_scatter(const moga_shape& s, const WsLayout& L, const void* Qp, const void* Kp,
+                                     const void* Vp, const int32_t* offsets, const int32_t* perm,
+                                     const float* gate, void* O, char* ws, cudaStream_t st);
+
 #define MOGA_CUDA_OK(expr)                                   \
   do {                                                       \
     cudaError_t e__ = (expr);                                \
