@@ -114,13 +114,24 @@ struct Shared {   // indices into the mbarrier array
   int q_full, q_empty, k_full, k_empty, v_full, v_empty, s_full, p_full, o_full, o_empty;
 };
 
+// Output placement.  perm == nullptr: rows stay in sorted order, Op is [B*H, T, D].
+// Otherwise (top-1 routing) the epilogue is the gated inverse permutation of Eq. 5: sorted
+// row p of batch item b goes to token perm[b, p] of O (element strides sb, sh, sn),
+// multiplied by gate[b, token] in fp32 before the one rounding to bf16.
+struct Scatter {
+  const int32_t* perm;
+  const float* gate;
+  long long sb, sh, sn;
+  int N;
+};
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                  const __grid_constant__ CUtensorMap mapV, const int32_t* __restrict__ offsets,
                  const int32_t* __restrict__ order, const int32_t* __restrict__ prefix,
                  __nv_bfloat16* __restrict__ Op, float* __restrict__ lse, uint32_t* header, int T, int H,
-                 int M, int BM, float scale_log2, float scale) {
+                 int M, int BM, float scale_log2, float scale, const Scatter sc) {
   using C = Cfg<D>;
   constexpr int NS = C::NS;
   extern __shared__ unsigned char smem_raw[];
@@ -415,7 +426,11 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       if (!ok) break;
       ++n_o;
       tc_fence_after();
-      const float inv_l = 1.f / l;
+      float inv_l = 1.f / l;
+      if (sc.perm != nullptr && tile_row0 + r < it.hi) {
+        const int b = it.bh / H;
+        inv_l *= sc.gate[(size_t)b * sc.N + sc.perm[(size_t)b * T + tile_row0 + r]];
+      }
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
         uint32_t oreg[32];
@@ -444,12 +459,26 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       if (!ok) break;
       constexpr int kChunks = D * 2 / 16;   // 16-byte chunks per row
       const int t = threadIdx.x - (4 + 4 * x) * 32;
+      if (sc.perm == nullptr) {
 #pragma unroll 4
-      for (int id = t; id < kTileM * kChunks; id += kTileM) {
-        const int row = id / kChunks, chunk = id % kChunks;
-        if (tile_row0 + row < it.hi) {
-          const uint4 val = *reinterpret_cast<const uint4*>(stage + row * (D * 2) + ((chunk ^ (row & 7)) * 16));
-          *reinterpret_cast<uint4*>(Op + ((size_t)it.bh * T + tile_row0 + row) * D + chunk * 8) = val;
+        for (int id = t; id < kTileM * kChunks; id += kTileM) {
+          const int row = id / kChunks, chunk = id % kChunks;
+          if (tile_row0 + row < it.hi) {
+            const uint4 val = *reinterpret_cast<const uint4*>(stage + row * (D * 2) + ((chunk ^ (row & 7)) * 16));
+            *reinterpret_cast<uint4*>(Op + ((size_t)it.bh * T + tile_row0 + row) * D + chunk * 8) = val;
+          }
+        }
+      } else {
+        const int b = it.bh / H, h = it.bh % H;
+        __nv_bfloat16* obase = Op + b * sc.sb + h * sc.sh;
+        const int32_t* prow = sc.perm + (size_t)b * T + tile_row0;
+#pragma unroll 4
+        for (int id = t; id < kTileM * kChunks; id += kTileM) {
+          const int row = id / kChunks, chunk = id % kChunks;
+          if (tile_row0 + row < it.hi) {
+            const uint4 val = *reinterpret_cast<const uint4*>(stage + row * (D * 2) + ((chunk ^ (row & 7)) * 16));
+            *reinterpret_cast<uint4*>(obase + (long long)prow[row] * sc.sn + chunk * 8) = val;
+          }
         }
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -488,7 +517,8 @@ bool make_map(CUtensorMap* map, const void* ptr, int D, long long T, long long B
 
 template <int D>
 moga_status launch(const moga_shape& s, const WsLayout& L, const void* Qp, const void* Kp, const void* Vp,
-                   const int32_t* offsets, void* Op, float* lse, char* ws, cudaStream_t st) {
+                   const int32_t* offsets, void* Op, float* lse, char* ws, const Scatter& sc,
+                   cudaStream_t st) {
   const long long T = (long long)s.N * s.k;
   CUtensorMap mq, mk, mv;
   if (!make_map(&mq, Qp, D, T, (long long)s.B * s.H) || !make_map(&mk, Kp, D, T, (long long)s.B * s.H) ||
@@ -512,7 +542,7 @@ moga_status launch(const moga_shape& s, const WsLayout& L, const void* Qp, const
   const float log2e = 1.4426950408889634f;
   kern<<<grid, kThreads, Cfg<D>::kDynSmem, st>>>(mq, mk, mv, offsets, order, prefix,
                                                   static_cast<__nv_bfloat16*>(Op), lse, header, (int)T, s.H,
-                                                  s.M, s.B * s.M, s.scale * log2e, s.scale);
+                                                  s.M, s.B * s.M, s.scale * log2e, s.scale, sc);
   MOGA_CUDA_OK(cudaGetLastError());
   return MOGA_OK;
 }
@@ -523,8 +553,19 @@ moga_status launch_attn_bf16(const moga_shape& s, const WsLayout& L, const void*
                              const void* Vp, const int32_t* offsets, void* Op, float* lse, char* ws,
                              cudaStream_t st) {
   if ((long long)s.N * s.k == 0) return MOGA_OK;
-  if (s.D == 128) return launch<128>(s, L, Qp, Kp, Vp, offsets, Op, lse, ws, st);
-  return launch<64>(s, L, Qp, Kp, Vp, offsets, Op, lse, ws, st);
+  const Scatter none{nullptr, nullptr, 0, 0, 0, 0};
+  if (s.D == 128) return launch<128>(s, L, Qp, Kp, Vp, offsets, Op, lse, ws, none, st);
+  return launch<64>(s, L, Qp, Kp, Vp, offsets, Op, lse, ws, none, st);
+}
+
+moga_status launch_attn_bf16_scatter(const moga_shape& s, const WsLayout& L, const void* Qp, const void* Kp,
+                                     const void* Vp, const int32_t* offsets, const int32_t* perm,
+                                     const float* gate, void* O, char* ws, cudaStream_t st) {
+  if ((long long)s.N * s.k == 0) return MOGA_OK;
+  const Strides q = qkv_strides(s);
+  const Scatter sc{perm, gate, q.b, q.h, q.n, s.N};
+  if (s.D == 128) return launch<128>(s, L, Qp, Kp, Vp, offsets, O, nullptr, ws, sc, st);
+  return launch<64>(s, L, Qp, Kp, Vp, offsets, O, nullptr, ws, sc, st);
 }
 
 }  // namespace moga
