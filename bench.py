@@ -35,7 +35,18 @@ from paper_2510_18692_b200.inputs import CONFIGS, make_inputs, useful_flops  # n
 
 METRIC = "MoGA fwd effective TFLOP/s (bf16)"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-KERNELS_PER_FORWARD = 9   # weight split, route, 3 sort kernels, gather, attention schedule, attention, unpermute
+# DRAM bytes of the attention kernel / its algorithmic bytes, from the ncu capture of the current
+# kernel summarised in profiles/attn_bf16_kernel_clip_bf16_ncu_full.md (traffic grows with T*H).
+ATTN_TRAFFIC_RATIO = 0.958
+
+
+def kernels_per_forward(cfg):
+    """Kernels one moga_forward launches: router (bf16: weight split + tensor-core router; fp32: one
+    ALU kernel), 3 sort kernels, gather, attention (bf16: schedule + attention), and the gated
+    unpermute unless the bf16 top-1 attention epilogue already wrote token order."""
+    if cfg.dtype == "bf16":
+        return 2 + 3 + 1 + 2 + (1 if cfg.k > 1 else 0)
+    return 1 + 3 + 1 + 1 + 1
 
 
 def load_peaks():
@@ -197,6 +208,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--stage", default="all", choices=["all", "route"],
+                    help="'route' times moga_route alone on the config's X (a small resident set, for profiling)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = CONFIGS[args.config]
@@ -215,6 +228,8 @@ def main():
     from paper_2510_18692_b200 import binding as mb   # raises if the CUDA library is missing
 
     cfg = cfg.with_(seed=cfg.seed + 100 * rank)       # every rank works on its own layer
+    if args.stage == "route":
+        return run_route_only(mb, cfg, dev, args)
     inp = make_inputs(cfg, device=dev)
     sh = mb.make_shape(cfg)
     ws = mb.alloc_workspace(mb.moga_workspace_bytes(sh), dev)
@@ -295,11 +310,14 @@ def main():
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic", "config": config_dict(cfg),
         "ms_per_layer_head_batch": ms / (cfg.B * cfg.H), "useful_tflop_per_step": flops / 1e12,
         "group_sizes": {"min": int(sizes.min()), "max": int(sizes.max()), "empty": int((sizes == 0).sum())},
-        "stages": stages_out, "gpu_launches": KERNELS_PER_FORWARD * args.steps, "clocks": clk,
+        "stages": stages_out, "gpu_launches": kernels_per_forward(cfg) * args.steps, "clocks": clk,
         "roofline": {"kernel": "moga_group_attn (tcgen05 varlen attention)", "bound": "tensor",
                      "achieved": attn_tflops, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                      "frac": attn_tflops / peaks["bf16_tflops_sustained"],
-                     "peak_source": f"{peaks['source']} sustained bf16 GEMM", "traffic": None},
+                     "peak_source": f"{peaks['source']} sustained bf16 GEMM",
+                     "frac_of_burst_peak": attn_tflops / peaks["bf16_tflops"],
+                     "traffic": ATTN_TRAFFIC_RATIO * 4.0 * tok * cfg.k * cfg.H * cfg.D * es if cfg.dtype == "bf16" else None,
+                     "traffic_unit": "bytes per launch (ncu dram bytes of the clip_bf16 capture, scaled by T*H)"},
     }
 
     if rank == 0 and not args.no_e2e:
@@ -320,6 +338,32 @@ def main():
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(out))
+    return 0
+
+
+def run_route_only(mb, cfg, dev, args):
+    """moga_route alone through the C ABI: X, W_r and the routing outputs are all that is resident."""
+    inp = make_inputs(cfg, device=dev, heads=[])
+    sh = mb.make_shape(cfg)
+    ws = mb.alloc_workspace(mb.moga_scratch_bytes(sh), dev)
+    gid = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.int32, device=dev)
+    gate = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.float32, device=dev)
+    for _ in range(args.warmup):
+        mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], gid, gate, None, ws)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(args.steps):
+        mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], gid, gate, None, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    es = 2 if cfg.dtype == "bf16" else 4
+    by = cfg.B * cfg.N * (cfg.C * es + cfg.k * 8)
+    peaks = load_peaks()
+    print(json.dumps({"stage": "route", "config": config_dict(cfg), "ms": ms, "GB/s": by / ms / 1e6,
+                      "frac_hbm": by / ms / 1e6 / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                      "device_status": mb.moga_last_device_status(ws)[0]}))
     return 0
 
 
