@@ -140,3 +140,25 @@ def forward(X, Wr, bias, Q, K, V, k, gate_mode, scale):
     if rc:
         raise ValueError(f"moga_oracle_forward rc={rc}")
     return dict(O=O, gid=gid, gate=gate, offsets=offsets, perm=perm, inv=inv)
+
+
+def balance_stats(gid, gate, M, alpha):
+    """Group-balancing loss of Eq. 6-8, written out per batch item in fp64.
+
+    F[b,i] = (assignments of item b to group i) / N (Eq. 7), P[b,i] = (1/N) * sum of the
+    routing probabilities (gates) of those assignments (Eq. 8: the sum runs over the tokens
+    routed to i only), loss[b] = alpha * M * sum_i F_i P_i (Eq. 6).  The paper states it for
+    top-1; with k > 1 every (token, slot) assignment counts once.
+    Returns F [B,M], P [B,M], loss [B], all float64."""
+    gid = np.asarray(gid)
+    gate = np.asarray(gate, dtype=np.float64)
+    B, N, k = gid.shape
+    F = np.zeros((B, M))
+    P = np.zeros((B, M))
+    for b in range(B):
+        for i in range(M):
+            sel = gid[b] == i
+            F[b, i] = sel.sum() / N
+            P[b, i] = gate[b][sel].sum() / N
+    loss = alpha * M * (F * P).sum(axis=1)
+    return F, P, loss

@@ -239,3 +239,36 @@ def test_balanced_flops_are_one_over_m():
     from paper_2510_18692_b200.inputs import useful_flops
     N, M, H, D = 4096, 8, 2, 64
     assert useful_flops([N // M] * M, H, D) == pytest.approx(useful_flops([N], H, D) / M)
+
+
+# ----------------------------------------------------------------------------- Eq. 6-8
+def test_balance_loss_closed_forms_and_brute_force():
+    """Eq. 6-8.  Uniform top-1 assignment with a constant probability p gives alpha * p
+    (F_i = 1/M, P_i = p/M); all tokens in one group gives alpha * M * p; among assignments
+    with equal probabilities the uniform one attains the minimum (the paper's remark after
+    Eq. 8); a pure-Python loop over tokens reproduces F, P and the loss on random input."""
+    M, N, alpha, p = 5, 1000, 0.1, 0.37
+    gid = (np.arange(N) % M).astype(np.int32).reshape(1, N, 1)
+    gate = np.full((1, N, 1), p)
+    F, P, loss = oracle.balance_stats(gid, gate, M, alpha)
+    assert np.allclose(F, 1.0 / M) and np.allclose(P, p / M) and np.isclose(loss[0], alpha * p)
+    F, P, loss = oracle.balance_stats(np.full((1, N, 1), 3, np.int32), gate, M, alpha)
+    assert np.isclose(loss[0], alpha * M * p) and F[0, 3] == 1.0 and F[0].sum() == 1.0
+    rng = np.random.default_rng(0)
+    for _ in range(20):                      # any other split of the tokens costs more
+        gid_r = rng.integers(0, M, (1, N, 1)).astype(np.int32)
+        assert oracle.balance_stats(gid_r, gate, M, alpha)[2][0] >= alpha * p - 1e-15
+    # brute force, k = 2, two batch items
+    B, N, k = 2, 57, 2
+    gid = np.stack([np.stack([rng.choice(M, k, replace=False) for _ in range(N)]) for _ in range(B)]).astype(np.int32)
+    gate = rng.random((B, N, k))
+    F, P, loss = oracle.balance_stats(gid, gate, M, 0.25)
+    for b in range(B):
+        f, q = [0.0] * M, [0.0] * M
+        for n in range(N):
+            for j in range(k):
+                f[gid[b, n, j]] += 1.0 / N
+                q[gid[b, n, j]] += gate[b, n, j] / N
+        assert np.allclose(F[b], f, rtol=0, atol=1e-12) and np.allclose(P[b], q, rtol=0, atol=1e-12)
+        assert abs(loss[b] - 0.25 * M * sum(x * y for x, y in zip(f, q))) <= 1e-12
+        assert abs(F[b].sum() - k) <= 1e-12
