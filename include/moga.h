@@ -101,6 +101,20 @@ moga_status moga_route(const moga_shape* s, const void* X, const float* Wr, cons
                        void* stream);
 
 /*
+ * Group-balancing statistics of Eq. 6-8 from a routing result (gid, gate as written by
+ * moga_route), per batch item b: F[b,i] = (assignments to group i) / N (Eq. 7),
+ * P[b,i] = (1/N) * sum of the gates of those assignments (Eq. 8: the routing probability
+ * of the chosen group, summed over the tokens routed to i only) and
+ * loss[b] = alpha * M * sum_i F[b,i] P[b,i] (Eq. 6).  The paper states them for top-1;
+ * with k > 1 every (token, slot) assignment counts once.  F, P: float [B, M]; loss: float
+ * [B]; device pointers.  Sums are taken in a fixed order (fp32 inside a block of 4,096
+ * assignments, fp64 across blocks), so results are reproducible bit for bit.
+ * ws: at least moga_scratch_bytes.  N = 0 is MOGA_ERR_INVALID_ARG.
+ */
+moga_status moga_balance_stats(const moga_shape* s, const int32_t* gid, const float* gate, float alpha,
+                               float* F, float* P, float* loss, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * "permute" of Alg. 1 line 2.  Stable counting sort of the N*k assignments of each
  * batch item by group (ascending token index inside a group): writes perm, inv,
  * offsets.  If Qp, Kp and Vp are all non-NULL the rows of Q, K, V are gathered

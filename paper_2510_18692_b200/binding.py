@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libmoga.so")
 
 EXPORTS = ("moga_workspace_bytes", "moga_scratch_bytes", "moga_status_string", "moga_route",
            "moga_permute", "moga_group_attn", "moga_unpermute", "moga_forward",
-           "moga_last_device_status", "moga_sort_static")
+           "moga_last_device_status", "moga_sort_static", "moga_balance_stats")
 
 MOGA_F32, MOGA_BF16 = 0, 1
 MOGA_ROUTE_AUTO, MOGA_ROUTE_ALU = 0, 1
@@ -95,6 +95,12 @@ def moga_route(shape, X, Wr, bias, gid, gate, logits=None, ws=None):
     _check(lib.moga_route(ctypes.byref(shape), _ptr(X), _ptr(Wr), _ptr(bias), _ptr(gid), _ptr(gate),
                           _ptr(logits), _ptr(ws), ctypes.c_size_t(0 if ws is None else ws.numel()),
                           _stream()), "moga_route")
+
+
+def moga_balance_stats(shape, gid, gate, alpha, F, P, loss, ws):
+    _check(lib.moga_balance_stats(ctypes.byref(shape), _ptr(gid), _ptr(gate), ctypes.c_float(alpha), _ptr(F),
+                                  _ptr(P), _ptr(loss), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()),
+           "moga_balance_stats")
 
 
 def moga_permute(shape, gid, Q, K, V, perm, inv, offsets, Qp, Kp, Vp, ws):

@@ -106,6 +106,21 @@ moga_status moga_route(const moga_shape* s, const void* X, const float* Wr, cons
   return launch_route(*s, X, Wr, bias, gid, gate, logits, cs);
 }
 
+moga_status moga_balance_stats(const moga_shape* s, const int32_t* gid, const float* gate, float alpha,
+                               float* F, float* P, float* loss, void* ws, size_t ws_bytes, void* stream) {
+  moga_status st;
+  if (!check_shape(s, &st)) return st;
+  if (!PTR_OK(gid) || !PTR_OK(gate) || F == nullptr || P == nullptr || loss == nullptr ||
+      (reinterpret_cast<uintptr_t>(F) & 3u) || (reinterpret_cast<uintptr_t>(P) & 3u) ||
+      (reinterpret_cast<uintptr_t>(loss) & 3u) || !(alpha == alpha))
+    return MOGA_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(*s);
+  if (!check_ws(ws, ws_bytes, L.scratch_end, &st)) return st;
+  if (s->N == 0) return MOGA_ERR_INVALID_ARG;     // the fractions of Eq. 7-8 divide by N
+  return launch_balance_stats(*s, L, gid, gate, alpha, F, P, loss, static_cast<char*>(ws),
+                              static_cast<cudaStream_t>(stream));
+}
+
 moga_status moga_permute(const moga_shape* s, const int32_t* gid, const void* Q, const void* K,
                          const void* V, int32_t* perm, int32_t* inv, int32_t* offsets, void* Qp,
                          void* Kp, void* Vp, void* ws, size_t ws_bytes, void* stream) {

@@ -26,6 +26,7 @@ struct WsLayout {
   size_t sort_hist;   // int32 [B, nblk, M]   per-block histograms, then bases
   size_t sched;       // int32 [B, 3, M+1]    attention schedule (order, tile prefix, ...)
   size_t wsplit;      // bf16 [3, MP, C]      router weight split into three bf16 parts (MP <= 64)
+  size_t stats;       // int32 + float [B, nblk, M] per-block counts and gate sums (Eq. 6-8)
   size_t scratch_end; // == moga_scratch_bytes
   size_t gid, gate, perm, inv, offsets;  // routing results
   size_t Qp, Kp, Vp, Op;                 // permuted tensors
@@ -46,6 +47,7 @@ inline WsLayout ws_layout(const moga_shape& s) {
   L.sort_hist = off;   off = align_up(off + sizeof(int32_t) * (size_t)s.B * L.nblk * s.M, kWsAlign);
   L.sched = off;       off = align_up(off + sizeof(int32_t) * (size_t)s.B * 4 * (s.M + 1) + 64, kWsAlign);
   L.wsplit = off;      off = align_up(off + sizeof(uint16_t) * 3 * (size_t)kMaxM * s.C, kWsAlign);
+  L.stats = off;       off = align_up(off + 2 * sizeof(int32_t) * (size_t)s.B * L.nblk * s.M, kWsAlign);
   L.scratch_end = off;
   L.gid = off;         off = align_up(off + sizeof(int32_t) * (size_t)s.B * T, kWsAlign);
   L.gate = off;        off = align_up(off + sizeof(float) * (size_t)s.B * T, kWsAlign);
@@ -79,6 +81,8 @@ moga_status launch_route(const moga_shape& s, const void* X, const float* Wr, co
 moga_status launch_route_mma(const moga_shape& s, const WsLayout& L, const void* X, const float* Wr,
                              const float* bias, int32_t* gid, float* gate, float* logits, char* ws,
                              cudaStream_t st);
+moga_status launch_balance_stats(const moga_shape& s, const WsLayout& L, const int32_t* gid, const float* gate,
+                                 float alpha, float* F, float* P, float* loss, char* ws, cudaStream_t st);
 moga_status launch_sort(const moga_shape& s, const WsLayout& L, const int32_t* gid, int32_t* perm,
                         int32_t* inv, int32_t* offsets, char* ws, cudaStream_t st);
 moga_status launch_gather(const moga_shape& s, const int32_t* perm, const void* Q, const void* K,

@@ -288,3 +288,31 @@ def test_group_attn_growing_scores_bf16(mb, grow):
         s = torch.einsum("bhnd,bhmd->bhnm", q[:, :, lo:hi], k_[:, :, lo:hi]) * scale
         ref = torch.logsumexp(s, -1)
         assert (lse[:, :, lo:hi].double().cpu() - ref).abs().max().item() <= 2e-2
+
+
+@pytest.mark.parametrize("B,N,M,k,skew", [(1, 5000, 8, 1, False), (2, 9001, 16, 2, False), (1, 40000, 64, 2, True),
+                                          (1, 1, 4, 1, False), (3, 4097, 1, 1, False)])
+def test_balance_stats(mb, B, N, M, k, skew):
+    """Eq. 6-8 from a routing result against the oracle, and reproducible bit for bit."""
+    cfg = _cfg(B=B, N=N, M=M, k=k, dtype="bf16")
+    gid_np = _random_gid(B, N, M, k, seed=N + 1, skew=skew) if k <= M else None
+    rng = np.random.default_rng(N)
+    gate_np = rng.random((B, N, k)).astype(np.float32)
+    gid, gate = torch.from_numpy(gid_np).cuda(), torch.from_numpy(gate_np).cuda()
+    sh = mb.make_shape(cfg)
+    ws = mb.alloc_workspace(mb.moga_scratch_bytes(sh))
+    outs = []
+    for _ in range(2):
+        F = torch.empty(B, M, device="cuda")
+        P = torch.empty(B, M, device="cuda")
+        loss = torch.empty(B, device="cuda")
+        mb.moga_balance_stats(sh, gid, gate, 0.1, F, P, loss, ws)
+        torch.cuda.synchronize()
+        outs.append((F, P, loss))
+    for a, b in zip(outs[0], outs[1]):
+        assert torch.equal(a, b)
+    oF, oP, oloss = oracle.balance_stats(gid_np, gate_np, M, 0.1)
+    F, P, loss = (t.double().cpu().numpy() for t in outs[0])
+    assert np.abs(F - oF).max() <= 1e-7                        # integer counts / N, rounded once to fp32
+    assert np.abs(P - oP).max() <= 2e-6 * max(1.0, oP.max())
+    assert np.abs(loss - oloss).max() <= 2e-6 * max(1.0, oloss.max())
