@@ -162,3 +162,68 @@ def balance_stats(gid, gate, M, alpha):
             P[b, i] = gate[b][sel].sum() / N
     loss = alpha * M * (F * P).sum(axis=1)
     return F, P, loss
+
+
+# ----------------------------------------------------------------------------- static groups (STGA)
+def stga_groups(F, Hh, Ww, wh, ww, shot_starts, tg, augment=True):
+    """Static spatial-temporal groups of Sec. 3.2 ("Spatial-Temporal Group Attention").
+
+    The latent video has F frames of Hh x Ww tokens, token index (f*Hh + y)*Ww + x.  Space is
+    cut into wh x ww fixed windows, each shot (frames [shot_starts[s], shot_starts[s+1])) into
+    runs of at most tg consecutive frames; frames of different shots never share a group.
+    A group is (shot, run, window); its queries are its own tokens.  Its keys/values are the
+    same tokens and, with ``augment``, the tokens of the same window in the last latent frame
+    of the previous shot (for the first run of a shot) and in the first latent frame of the
+    next shot (for the last run of a shot): the paper's "two latent frames from adjacent
+    shots", keys/values only.  Returns two lists of int arrays (query tokens, key tokens) in
+    the order (shot, run, window), tokens ascending, the augmenting frames before / after."""
+    starts = list(shot_starts) + [F]
+    assert starts[0] == 0 and all(a < b for a, b in zip(starts, starts[1:]))
+
+    def window_tokens(f, wy, wx):
+        return [(f * Hh + y) * Ww + x for y in range(Hh) if y * wh // Hh == wy
+                for x in range(Ww) if x * ww // Ww == wx]
+
+    q_groups, kv_groups = [], []
+    for s in range(len(starts) - 1):
+        f0, f1 = starts[s], starts[s + 1]
+        runs = [(a, min(a + tg, f1)) for a in range(f0, f1, tg)]
+        for r, (a, b) in enumerate(runs):
+            for wy in range(wh):
+                for wx in range(ww):
+                    own = [t for f in range(a, b) for t in window_tokens(f, wy, wx)]
+                    if not own:
+                        continue
+                    before = window_tokens(f0 - 1, wy, wx) if augment and r == 0 and s > 0 else []
+                    after = (window_tokens(f1, wy, wx)
+                             if augment and r == len(runs) - 1 and s < len(starts) - 2 else [])
+                    q_groups.append(np.array(own, np.int64))
+                    kv_groups.append(np.array(before + own + after, np.int64))
+    return q_groups, kv_groups
+
+
+def frame_groups(F, Hh, Ww):
+    """Per-frame attention of Sec. 3.2: one group per latent frame, keys = queries."""
+    g = [np.arange(f * Hh * Ww, (f + 1) * Hh * Ww, dtype=np.int64) for f in range(F)]
+    return g, g
+
+
+def static_group_attn(Q, K, V, q_groups, kv_groups, scale):
+    """Eq. 1 inside caller-given groups whose query and key/value sets may differ:
+    O[b,h,n,:] = softmax_m(scale * <Q[b,h,n], K[b,h,m]>) V[b,h,m] over the keys m of the group
+    that holds query n.  Q,K,V [B,H,N,D] (exact float32 copies of the inputs); fp64 result
+    [B,H,N,D]; tokens in no query group stay zero."""
+    Q, K, V = (np.asarray(a, dtype=np.float64) for a in (Q, K, V))
+    O = np.zeros_like(Q)
+    for qi, ki in zip(q_groups, kv_groups):
+        s = np.einsum("bhnd,bhmd->bhnm", Q[:, :, qi], K[:, :, ki]) * scale
+        s = s - s.max(axis=-1, keepdims=True)
+        p = np.exp(s)
+        p /= p.sum(axis=-1, keepdims=True)
+        O[:, :, qi] = np.einsum("bhnm,bhmd->bhnd", p, V[:, :, ki])
+    return O
+
+
+def mean3(a, b, c):
+    """Sec. 3.2: a token's output is the mean of its dynamic (MoGA) and two static group outputs."""
+    return (np.asarray(a, np.float64) + np.asarray(b, np.float64) + np.asarray(c, np.float64)) / 3.0

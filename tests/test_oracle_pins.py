@@ -272,3 +272,91 @@ def test_balance_loss_closed_forms_and_brute_force():
         assert np.allclose(F[b], f, rtol=0, atol=1e-12) and np.allclose(P[b], q, rtol=0, atol=1e-12)
         assert abs(loss[b] - 0.25 * M * sum(x * y for x, y in zip(f, q))) <= 1e-12
         assert abs(F[b].sum() - k) <= 1e-12
+
+
+# ----------------------------------------------------------------------------- Sec. 3.2 static groups
+def _token_coords(n, Hh, Ww):
+    return n // (Hh * Ww), (n // Ww) % Hh, n % Ww
+
+
+def test_stga_groups_against_the_membership_rule():
+    """The group lists against the rule of Sec. 3.2 stated per token pair: query n sees key m
+    iff both lie in the same window and either in the same run of the same shot, or m is in
+    the frame just across the shot boundary that n's run touches."""
+    F, Hh, Ww, wh, ww, tg = 9, 4, 6, 2, 3, 2
+    shots = [0, 3, 4]                                   # shots of 3, 1 and 5 frames
+    qg, kg = oracle.stga_groups(F, Hh, Ww, wh, ww, shots, tg)
+    N = F * Hh * Ww
+    seen = np.zeros(N, int)
+    keyset = {}
+    for qi, ki in zip(qg, kg):
+        seen[qi] += 1
+        assert len(set(ki.tolist())) == len(ki)
+        for n in qi:
+            keyset[int(n)] = set(ki.tolist())
+    assert np.all(seen == 1)                            # every token queries in exactly one group
+    bounds = shots + [F]
+    shot_of = lambda f: max(s for s in range(len(shots)) if bounds[s] <= f)
+    for n in range(N):
+        f, y, x = _token_coords(n, Hh, Ww)
+        s = shot_of(f)
+        run = (f - bounds[s]) // tg
+        last_run = (bounds[s + 1] - 1 - bounds[s]) // tg
+        want = set()
+        for m in range(N):
+            g, v, u = _token_coords(m, Hh, Ww)
+            if (v * wh // Hh, u * ww // Ww) != (y * wh // Hh, x * ww // Ww):
+                continue
+            same = shot_of(g) == s and (g - bounds[s]) // tg == run
+            prev_edge = run == 0 and s > 0 and g == bounds[s] - 1
+            next_edge = run == last_run and s < len(shots) - 1 and g == bounds[s + 1]
+            if same or prev_edge or next_edge:
+                want.add(m)
+        assert keyset[n] == want, n
+    # without augmentation keys = queries; a one-frame shot between two others gets both neighbours
+    q2, k2 = oracle.stga_groups(F, Hh, Ww, wh, ww, shots, tg, augment=False)
+    assert all(np.array_equal(a, b) for a, b in zip(q2, k2))
+    per_win = (Hh // wh) * (Ww // ww)
+    mid = [(a, b) for a, b in zip(qg, kg) if _token_coords(int(a[0]), Hh, Ww)[0] == 3]
+    assert all(len(b) - len(a) == 2 * per_win for a, b in mid)
+
+
+def test_static_group_attention_special_cases():
+    """One shot, one window, one run: the static group is the whole sequence and the result is
+    plain full attention (library routine).  Per-frame groups: each frame equals full
+    attention on that frame alone.  Keys-only augmentation: changing K/V of an augmenting
+    frame changes the neighbour shot's boundary group and nothing else."""
+    rng = np.random.default_rng(3)
+    F, Hh, Ww, D = 4, 3, 4, 8
+    N = F * Hh * Ww
+    Q, K, V = (rng.standard_normal((1, 2, N, D)).astype(np.float32) for _ in range(3))
+    scale = 1 / np.sqrt(D)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(Q).double(), torch.from_numpy(K).double(), torch.from_numpy(V).double(), scale=scale).numpy()
+    qg, kg = oracle.stga_groups(F, Hh, Ww, 1, 1, [0], F)
+    assert len(qg) == 1
+    assert np.abs(oracle.static_group_attn(Q, K, V, qg, kg, scale) - ref).max() < 1e-12
+    fq, fk = oracle.frame_groups(F, Hh, Ww)
+    Of = oracle.static_group_attn(Q, K, V, fq, fk, scale)
+    for f in range(F):
+        sl = slice(f * Hh * Ww, (f + 1) * Hh * Ww)
+        r = torch.nn.functional.scaled_dot_product_attention(
+            torch.from_numpy(Q[:, :, sl]).double(), torch.from_numpy(K[:, :, sl]).double(),
+            torch.from_numpy(V[:, :, sl]).double(), scale=scale).numpy()
+        assert np.abs(Of[:, :, sl] - r).max() < 1e-12
+    # two shots of two frames, one run each: frame 1 augments shot 1, frame 2 augments shot 0
+    qg, kg = oracle.stga_groups(F, Hh, Ww, 1, 2, [0, 2], 2)
+    O1 = oracle.static_group_attn(Q, K, V, qg, kg, scale)
+    K2, V2 = K.copy(), V.copy()
+    f0 = slice(0, Hh * Ww)                              # frame 0 augments nobody
+    K2[:, :, f0] += 1.0
+    V2[:, :, f0] -= 2.0
+    O2 = oracle.static_group_attn(Q, K2, V2, qg, kg, scale)
+    shot1 = slice(2 * Hh * Ww, N)
+    assert np.array_equal(O1[:, :, shot1], O2[:, :, shot1])          # shot 1 never sees frame 0
+    assert np.abs(O1[:, :, f0] - O2[:, :, f0]).max() > 1e-3
+    K3 = K.copy()
+    K3[:, :, Hh * Ww:2 * Hh * Ww] *= 1.5                # frame 1: last frame of shot 0, seen by shot 1
+    O3 = oracle.static_group_attn(Q, K3, V, qg, kg, scale)
+    assert np.abs(O1[:, :, shot1] - O3[:, :, shot1]).max() > 1e-4
+    assert np.abs(oracle.mean3(O1, O2, O3) - (O1 + O2 + O3) / 3).max() == 0
