@@ -166,6 +166,68 @@ moga_status moga_group_attn(const moga_shape* s, const void* Qp, const void* Kp,
                             size_t ws_bytes, void* stream);
 
 /*
+ * ---- Static groups: Sec. 3.2, "Spatial-Temporal Group Attention" -----------------------
+ * A token's visual-attention output is the mean of three group attentions: the routed one
+ * above and two with fixed groups (spatial window x run of frames inside a shot, and one
+ * group per latent frame).  The fixed groups are the same for every batch item and head,
+ * and a group's key/value set may be larger than its query set (boundary groups also see
+ * one latent frame of the adjacent shot).
+ */
+
+/*
+ * Host only, no CUDA call: the group lists of the spatial-temporal branch for a latent
+ * video of F frames of Hh x Ww tokens (token index (f*Hh + y)*Ww + x), wh x ww spatial
+ * windows (window of (y, x) = (y*wh/Hh, x*ww/Ww)), shots starting at the n_shots frames
+ * shot_starts[] (ascending, shot_starts[0] = 0), runs of at most tg frames inside a shot.
+ * Group order: shot, run, window.  Queries of a group: its own tokens, ascending.  Keys:
+ * with augment != 0 the same window of the previous shot's last frame (first run of a shot)
+ * and of the next shot's first frame (last run of a shot) are added before / after them.
+ * All pointers are HOST pointers and may be NULL (sizes only): q_idx [N] token at each
+ * query position, q_inv [N] query position of each token, q_offsets / kv_offsets [G+1],
+ * kv_idx [Tkv]; *G_out and *Tkv_out receive the counts (N = F*Hh*Ww, Tkv <= 3*N: size
+ * kv_idx from a first call with NULL lists).
+ */
+moga_status moga_stga_build(int32_t F, int32_t Hh, int32_t Ww, int32_t wh, int32_t ww,
+                            const int32_t* shot_starts, int32_t n_shots, int32_t tg, int32_t augment,
+                            int32_t* q_idx, int32_t* q_inv, int32_t* q_offsets, int32_t* kv_idx,
+                            int32_t* kv_offsets, int32_t* G_out, int32_t* Tkv_out);
+
+/*
+ * dst[b,h,p,:] = src[b,h,idx[p],:] for p < L: rows of src (strides from the shape, N rows)
+ * listed by the device array idx [L], shared by all batch items and heads, into the
+ * contiguous dst [B, H, L, D].  16-byte vector copies; no workspace.
+ */
+moga_status moga_gather_rows(const moga_shape* s, const int32_t* idx, int32_t L, const void* src, void* dst,
+                             void* stream);
+
+/* Bytes of ws moga_static_group_attn needs for G groups (host only; 0 if the shape is invalid). */
+size_t moga_static_scratch_bytes(const moga_shape* s, int32_t G);
+
+/*
+ * Eq. 1 inside caller-given groups: query rows [q_offsets[g], q_offsets[g+1]) of
+ * Qs [B, H, Tq, D] attend to key/value rows [kv_offsets[g], kv_offsets[g+1]) of
+ * Ks, Vs [B, H, Tkv, D]; the result goes to the same rows of Os [B, H, Tq, D]
+ * (lse [B, H, Tq] optional).  q_offsets, kv_offsets: device int32 [G+1], one list for all
+ * batch items and heads.  Same kernels as moga_group_attn (which is the case Tq = Tkv,
+ * q_offsets = kv_offsets per batch item).  Rows of a group without keys, and rows outside
+ * every group, are left untouched.  M and k of the shape are not used.
+ */
+moga_status moga_static_group_attn(const moga_shape* s, int32_t G, int32_t Tq, int32_t Tkv, const void* Qs,
+                                   const void* Ks, const void* Vs, const int32_t* q_offsets,
+                                   const int32_t* kv_offsets, void* Os, float* lse, void* ws,
+                                   size_t ws_bytes, void* stream);
+
+/*
+ * The mean of the three branch outputs (Sec. 3.2): O[b,h,n,:] = (A[b,h,n,:] +
+ * Bs[b,h,inv_b[n],:] + C[b,h,n,:]) / 3, summed in fp32 and rounded once.  A and O use the
+ * shape's strides (token order); Bs [B, H, N, D] is contiguous in the spatial-temporal
+ * branch's query order, inv_b [N] (device, NULL = identity) gives each token's position in
+ * it; C [B, H, N, D] is contiguous in token order (per-frame groups keep token order).
+ */
+moga_status moga_mean3(const moga_shape* s, const void* A, const void* Bs, const int32_t* inv_b,
+                       const void* C, void* O, void* stream);
+
+/*
  * "repermute" of Alg. 1 line 4 with the gate of Eq. 5:
  * O[b,h,n,:] = sum_j gate[b,n,j] * Op[b,h,inv[b,n,j],:], summed in fp32 in slot
  * order and rounded once.  No workspace.

@@ -19,7 +19,8 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libmoga.so")
 
 EXPORTS = ("moga_workspace_bytes", "moga_scratch_bytes", "moga_status_string", "moga_route",
            "moga_permute", "moga_group_attn", "moga_unpermute", "moga_forward",
-           "moga_last_device_status", "moga_sort_static", "moga_balance_stats")
+           "moga_last_device_status", "moga_sort_static", "moga_balance_stats", "moga_stga_build", "moga_gather_rows",
+           "moga_static_group_attn", "moga_mean3")
 
 MOGA_F32, MOGA_BF16 = 0, 1
 MOGA_ROUTE_AUTO, MOGA_ROUTE_ALU = 0, 1
@@ -49,6 +50,7 @@ if not os.path.exists(LIB_PATH):
 lib = ctypes.CDLL(LIB_PATH)
 lib.moga_workspace_bytes.restype = ctypes.c_size_t
 lib.moga_scratch_bytes.restype = ctypes.c_size_t
+lib.moga_static_scratch_bytes.restype = ctypes.c_size_t
 lib.moga_status_string.restype = ctypes.c_char_p
 for _n in EXPORTS[3:]:
     getattr(lib, _n).restype = ctypes.c_int
@@ -119,6 +121,48 @@ def moga_group_attn(shape, Qp, Kp, Vp, offsets, Op, lse, ws):
     _check(lib.moga_group_attn(ctypes.byref(shape), _ptr(Qp), _ptr(Kp), _ptr(Vp), _ptr(offsets),
                                _ptr(Op), _ptr(lse), _ptr(ws), ctypes.c_size_t(ws.numel()),
                                _stream()), "moga_group_attn")
+
+
+def moga_stga_build(F, Hh, Ww, wh, ww, shot_starts, tg, augment=True):
+    """Host-side group lists of the spatial-temporal branch: dict of numpy int32 arrays
+    q_idx, q_inv, q_offsets, kv_idx, kv_offsets (plus G, Tkv)."""
+    import numpy as np
+    shots = (ctypes.c_int32 * len(shot_starts))(*shot_starts)
+    G, Tkv = ctypes.c_int32(0), ctypes.c_int32(0)
+    null = ctypes.c_void_p(0)
+    args = (ctypes.c_int32(F), ctypes.c_int32(Hh), ctypes.c_int32(Ww), ctypes.c_int32(wh), ctypes.c_int32(ww),
+            shots, ctypes.c_int32(len(shot_starts)), ctypes.c_int32(tg), ctypes.c_int32(1 if augment else 0))
+    _check(lib.moga_stga_build(*args, null, null, null, null, null, ctypes.byref(G), ctypes.byref(Tkv)),
+           "moga_stga_build")
+    N = F * Hh * Ww
+    out = dict(q_idx=np.empty(N, np.int32), q_inv=np.empty(N, np.int32), q_offsets=np.empty(G.value + 1, np.int32),
+               kv_idx=np.empty(Tkv.value, np.int32), kv_offsets=np.empty(G.value + 1, np.int32))
+    p = lambda a: a.ctypes.data_as(ctypes.c_void_p)
+    _check(lib.moga_stga_build(*args, p(out["q_idx"]), p(out["q_inv"]), p(out["q_offsets"]), p(out["kv_idx"]),
+                               p(out["kv_offsets"]), ctypes.byref(G), ctypes.byref(Tkv)), "moga_stga_build")
+    out.update(G=G.value, Tkv=Tkv.value)
+    return out
+
+
+def moga_static_scratch_bytes(shape, G) -> int:
+    return int(lib.moga_static_scratch_bytes(ctypes.byref(shape), ctypes.c_int32(G)))
+
+
+def moga_gather_rows(shape, idx, src, dst):
+    _check(lib.moga_gather_rows(ctypes.byref(shape), _ptr(idx), ctypes.c_int32(idx.numel()), _ptr(src), _ptr(dst),
+                                _stream()), "moga_gather_rows")
+
+
+def moga_static_group_attn(shape, G, Tq, Tkv, Qs, Ks, Vs, q_offsets, kv_offsets, Os, lse, ws):
+    _check(lib.moga_static_group_attn(ctypes.byref(shape), ctypes.c_int32(G), ctypes.c_int32(Tq), ctypes.c_int32(Tkv),
+                                      _ptr(Qs), _ptr(Ks), _ptr(Vs), _ptr(q_offsets), _ptr(kv_offsets), _ptr(Os),
+                                      _ptr(lse), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()),
+           "moga_static_group_attn")
+
+
+def moga_mean3(shape, A, Bs, inv_b, C, O):
+    _check(lib.moga_mean3(ctypes.byref(shape), _ptr(A), _ptr(Bs), _ptr(inv_b), _ptr(C), _ptr(O), _stream()),
+           "moga_mean3")
 
 
 def moga_unpermute(shape, Op, inv, gate, O):

@@ -36,61 +36,84 @@ constexpr float kRowSumLimit = 1.0995116e12f;      // 2^40: a tile's row sum bey
 using namespace sm100;
 
 // ----------------------------------------------------------------------------- schedule
-// order[b*M + r]  : group with the r-th largest size in batch item b
-// prefix[b*M + r] : number of work items before (b, r); prefix[B*M] = total
-__global__ void attn_schedule_kernel(const int32_t* __restrict__ offsets, int32_t* __restrict__ order,
-                                     int32_t* __restrict__ prefix, int B, int M, int H) {
-  for (int idx = threadIdx.x; idx < B * M; idx += blockDim.x) {
-    const int b = idx / M, g = idx % M;
-    const int32_t* off = offsets + (size_t)b * (M + 1);
-    const int n = off[g + 1] - off[g];
-    int r = 0;
-    for (int o = 0; o < M; ++o) {
-      const int no = off[o + 1] - off[o];
-      r += (no > n) || (no == n && o < g);
+// The groups of one launch.  Group g of batch item b owns query rows
+// [q_off[b*stride + g], q_off[b*stride + g + 1]) of Q / O and key rows
+// [kv_off[b*stride + g], kv_off[b*stride + g + 1]) of K / V.  Routed groups (Alg. 1): q_off and
+// kv_off are the same array, stride = G + 1.  Static groups (Sec. 3.2): one list shared by
+// all batch items (stride 0), keys may be a superset of the queries.
+struct Groups {
+  const int32_t* q_off;
+  const int32_t* kv_off;
+  int stride;
+  int G;
+};
+
+constexpr int kRankLimit = 256;   // above this many groups per item the list keeps its order
+
+// order[b*G + r]  : group with the r-th largest cost (queries x keys) in batch item b
+// prefix[b*G + r] : number of work items before (b, r); prefix[B*G] = total
+// A group with queries but no keys gets no work item: its rows are left untouched.
+__global__ void attn_schedule_kernel(const Groups grp, int32_t* __restrict__ order, int32_t* __restrict__ prefix,
+                                     int B, int H) {
+  const int G = grp.G;
+  for (int idx = threadIdx.x; idx < B * G; idx += blockDim.x) {
+    const int b = idx / G, g = idx % G;
+    int r = g;
+    if (G <= kRankLimit) {
+      const int32_t* qo = grp.q_off + (size_t)b * grp.stride;
+      const int32_t* ko = grp.kv_off + (size_t)b * grp.stride;
+      const long long n = (long long)(qo[g + 1] - qo[g]) * (ko[g + 1] - ko[g]);
+      r = 0;
+      for (int o = 0; o < G; ++o) {
+        const long long no = (long long)(qo[o + 1] - qo[o]) * (ko[o + 1] - ko[o]);
+        r += (no > n) || (no == n && o < g);
+      }
     }
-    order[b * M + r] = g;
+    order[b * G + r] = g;
   }
   __syncthreads();
   if (threadIdx.x == 0) {
     int acc = 0;
-    for (int idx = 0; idx < B * M; ++idx) {
-      const int b = idx / M;
-      const int32_t* off = offsets + (size_t)b * (M + 1);
+    for (int idx = 0; idx < B * G; ++idx) {
+      const int b = idx / G;
       const int g = order[idx];
-      const int n = off[g + 1] - off[g];
+      const int nq = grp.q_off[(size_t)b * grp.stride + g + 1] - grp.q_off[(size_t)b * grp.stride + g];
+      const int nk = grp.kv_off[(size_t)b * grp.stride + g + 1] - grp.kv_off[(size_t)b * grp.stride + g];
       prefix[idx] = acc;
-      acc += ((n + kQBlock - 1) / kQBlock) * H;
+      if (nk > 0) acc += ((nq + kQBlock - 1) / kQBlock) * H;
     }
-    prefix[B * M] = acc;
+    prefix[B * G] = acc;
   }
 }
 
 struct Item {
-  int bh;        // b * H + h
-  int row0;      // first sorted position of the query block
-  int lo, hi;    // the group's range of sorted positions
+  int bh;          // b * H + h
+  int row0;        // first row of the query block
+  int qhi;         // end of the group's query rows
+  int klo, khi;    // the group's key rows
 };
 
-__device__ __forceinline__ Item decode_item(int w, const int32_t* __restrict__ offsets,
-                                            const int32_t* __restrict__ order,
-                                            const int32_t* __restrict__ prefix, int BM, int M, int H) {
-  int lo = 0, hi = BM;           // largest idx with prefix[idx] <= w
+__device__ __forceinline__ Item decode_item(int w, const Groups& grp, const int32_t* __restrict__ order,
+                                            const int32_t* __restrict__ prefix, int BG, int H) {
+  int lo = 0, hi = BG;           // largest idx with prefix[idx] <= w (entries without items are skipped)
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
     if (prefix[mid] <= w) lo = mid; else hi = mid;
   }
-  const int b = lo / M;
+  const int b = lo / grp.G;
   const int g = order[lo];
-  const int32_t* off = offsets + (size_t)b * (M + 1);
+  const int32_t* qo = grp.q_off + (size_t)b * grp.stride;
+  const int32_t* ko = grp.kv_off + (size_t)b * grp.stride;
   Item it;
-  it.lo = off[g];
-  it.hi = off[g + 1];
-  const int nqb = (it.hi - it.lo + kQBlock - 1) / kQBlock;
+  const int qlo = qo[g];
+  it.qhi = qo[g + 1];
+  it.klo = ko[g];
+  it.khi = ko[g + 1];
+  const int nqb = (it.qhi - qlo + kQBlock - 1) / kQBlock;
   const int local = w - prefix[lo];
   const int h = local / nqb, qb = local % nqb;
   it.bh = b * H + h;
-  it.row0 = it.lo + qb * kQBlock;
+  it.row0 = qlo + qb * kQBlock;
   return it;
 }
 
@@ -128,10 +151,10 @@ struct Scatter {
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
-                 const __grid_constant__ CUtensorMap mapV, const int32_t* __restrict__ offsets,
+                 const __grid_constant__ CUtensorMap mapV, const Groups grp,
                  const int32_t* __restrict__ order, const int32_t* __restrict__ prefix,
                  __nv_bfloat16* __restrict__ Op, float* __restrict__ lse, uint32_t* header, int T, int H,
-                 int M, int BM, float scale_log2, float scale, const Scatter sc) {
+                 int BG, float scale_log2, float scale, const Scatter sc) {
   using C = Cfg<D>;
   constexpr int NS = C::NS;
   extern __shared__ unsigned char smem_raw[];
@@ -148,7 +171,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total_items = prefix[BM];
+  const int total_items = prefix[BG];
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
@@ -213,9 +236,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       uint32_t nq[2] = {0, 0}, nkv = 0;
       bool ok = true;
       for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
-        const Item it = decode_item(w, offsets, order, prefix, BM, M, H);
-        const int ntiles = (it.hi - it.lo + kTileN - 1) / kTileN;
-        const bool validB = it.row0 + kTileM < it.hi;
+        const Item it = decode_item(w, grp, order, prefix, BG, H);
+        const int ntiles = (it.khi - it.klo + kTileN - 1) / kTileN;
+        const bool validB = it.row0 + kTileM < it.qhi;
         for (int x = 0; x < (validB ? 2 : 1) && ok; ++x) {
           ok = wait(Q_EMPTY + x, (nq[x] & 1u) ^ 1u, 1);
           if (!ok) break;
@@ -235,14 +258,14 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 #pragma unroll
           for (int bx = 0; bx < C::kBoxes; ++bx)
             tma_load_3d(sK + s * C::kTileBytes + bx * C::kBoxBytes, &mapK, bar(K_FULL + s), bx * 64,
-                        it.lo + j * kTileN, it.bh);
+                        it.klo + j * kTileN, it.bh);
           ok = wait(V_EMPTY + s, ph, 3);
           if (!ok) break;
           mbar_expect_tx(bar(V_FULL + s), C::kTileBytes);
 #pragma unroll
           for (int bx = 0; bx < C::kBoxes; ++bx)
             tma_load_3d(sV + s * C::kTileBytes + bx * C::kBoxBytes, &mapV, bar(V_FULL + s), bx * 64,
-                        it.lo + j * kTileN, it.bh);
+                        it.klo + j * kTileN, it.bh);
           ++nkv;
         }
       }
@@ -273,9 +296,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                  (accumulate || kk > 0) ? 1u : 0u);
       };
       for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
-        const Item it = decode_item(w, offsets, order, prefix, BM, M, H);
-        const int ntiles = (it.hi - it.lo + kTileN - 1) / kTileN;
-        const int nx = (it.row0 + kTileM < it.hi) ? 2 : 1;
+        const Item it = decode_item(w, grp, order, prefix, BG, H);
+        const int ntiles = (it.khi - it.klo + kTileN - 1) / kTileN;
+        const int nx = (it.row0 + kTileM < it.qhi) ? 2 : 1;
         // first S tiles
         for (int x = 0; x < nx && ok; ++x) {
           ok = wait(Q_FULL + x, nq[x] & 1u, 4);
@@ -342,9 +365,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     uint32_t n_s = 0, n_o = 0;
     bool ok = true;
     for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
-      const Item it = decode_item(w, offsets, order, prefix, BM, M, H);
-      if (x == 1 && !(it.row0 + kTileM < it.hi)) continue;
-      const int ntiles = (it.hi - it.lo + kTileN - 1) / kTileN;
+      const Item it = decode_item(w, grp, order, prefix, BG, H);
+      if (x == 1 && !(it.row0 + kTileM < it.qhi)) continue;
+      const int ntiles = (it.khi - it.klo + kTileN - 1) / kTileN;
       const int tile_row0 = it.row0 + x * kTileM;
       float m = -INFINITY, l = 0.f;
       for (int j = 0; j < ntiles && ok; ++j) {
@@ -360,7 +383,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         uint32_t preg[64];
         float alpha = 1.f, lsum;
         bool exact = (j == 0), rescale = false;
-        const int ncols = it.hi - it.lo - j * kTileN;     // valid keys in this tile (may exceed 128)
+        const int ncols = it.khi - it.klo - j * kTileN;     // valid keys in this tile (may exceed 128)
         while (true) {
           uint32_t sreg[128];
 #pragma unroll
@@ -427,7 +450,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       ++n_o;
       tc_fence_after();
       float inv_l = 1.f / l;
-      if (sc.perm != nullptr && tile_row0 + r < it.hi) {
+      if (sc.perm != nullptr && tile_row0 + r < it.qhi) {
         const int b = it.bh / H;
         inv_l *= sc.gate[(size_t)b * sc.N + sc.perm[(size_t)b * T + tile_row0 + r]];
       }
@@ -452,7 +475,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       }
       tc_fence_before();
       mbar_arrive(bar(O_EMPTY + x));        // TMEM O (and S) of this tile may be overwritten
-      if (lse != nullptr && tile_row0 + r < it.hi)
+      if (lse != nullptr && tile_row0 + r < it.qhi)
         lse[(size_t)it.bh * T + tile_row0 + r] = m * scale + __logf(l);
       mbar_arrive(bar(STG_FULL + x));          // all 128 rows staged (bounded wait, no bar.sync)
       ok = wait(STG_FULL + x, (n_o & 1u) ^ 1u, 12);
@@ -463,7 +486,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 #pragma unroll 4
         for (int id = t; id < kTileM * kChunks; id += kTileM) {
           const int row = id / kChunks, chunk = id % kChunks;
-          if (tile_row0 + row < it.hi) {
+          if (tile_row0 + row < it.qhi) {
             const uint4 val = *reinterpret_cast<const uint4*>(stage + row * (D * 2) + ((chunk ^ (row & 7)) * 16));
             *reinterpret_cast<uint4*>(Op + ((size_t)it.bh * T + tile_row0 + row) * D + chunk * 8) = val;
           }
@@ -475,7 +498,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 #pragma unroll 4
         for (int id = t; id < kTileM * kChunks; id += kTileM) {
           const int row = id / kChunks, chunk = id % kChunks;
-          if (tile_row0 + row < it.hi) {
+          if (tile_row0 + row < it.qhi) {
             const uint4 val = *reinterpret_cast<const uint4*>(stage + row * (D * 2) + ((chunk ^ (row & 7)) * 16));
             *reinterpret_cast<uint4*>(obase + (long long)prow[row] * sc.sn + chunk * 8) = val;
           }
@@ -515,19 +538,27 @@ bool make_map(CUtensorMap* map, const void* ptr, int D, long long T, long long B
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// One launch: B*H heads, groups grp, Q / O with Tq rows and K / V with Tkv rows per head.
+struct Problem {
+  int B, H;
+  long long Tq, Tkv;
+  float scale;
+  const void *Q, *K, *V;
+  void* O;
+  float* lse;
+  Groups grp;
+  int32_t *order, *prefix;   // scratch: B*G and B*G + 1 int32
+  uint32_t* header;          // device status word
+  Scatter sc;
+};
+
 template <int D>
-moga_status launch(const moga_shape& s, const WsLayout& L, const void* Qp, const void* Kp, const void* Vp,
-                   const int32_t* offsets, void* Op, float* lse, char* ws, const Scatter& sc,
-                   cudaStream_t st) {
-  const long long T = (long long)s.N * s.k;
+moga_status launch(const Problem& p, cudaStream_t st) {
   CUtensorMap mq, mk, mv;
-  if (!make_map(&mq, Qp, D, T, (long long)s.B * s.H) || !make_map(&mk, Kp, D, T, (long long)s.B * s.H) ||
-      !make_map(&mv, Vp, D, T, (long long)s.B * s.H))
+  const long long BH = (long long)p.B * p.H;
+  if (!make_map(&mq, p.Q, D, p.Tq, BH) || !make_map(&mk, p.K, D, p.Tkv, BH) || !make_map(&mv, p.V, D, p.Tkv, BH))
     return MOGA_ERR_CUDA;
-  int32_t* order = reinterpret_cast<int32_t*>(ws + L.sched);
-  int32_t* prefix = order + (size_t)s.B * s.M;
-  uint32_t* header = reinterpret_cast<uint32_t*>(ws + L.header);
-  attn_schedule_kernel<<<1, 256, 0, st>>>(offsets, order, prefix, s.B, s.M, s.H);
+  attn_schedule_kernel<<<1, 1024, 0, st>>>(p.grp, p.order, p.prefix, p.B, p.H);
   MOGA_CUDA_OK(cudaGetLastError());
   static int num_sms = 0;
   if (num_sms == 0) {
@@ -537,14 +568,27 @@ moga_status launch(const moga_shape& s, const WsLayout& L, const void* Qp, const
   }
   auto kern = attn_bf16_kernel<D>;
   MOGA_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::kDynSmem));
-  const long long max_items = ((T + kQBlock - 1) / kQBlock + s.M) * (long long)s.B * s.H;
+  const long long max_items = ((p.Tq + kQBlock - 1) / kQBlock + p.grp.G) * BH;
   const int grid = (int)(max_items < num_sms ? max_items : num_sms);
   const float log2e = 1.4426950408889634f;
-  kern<<<grid, kThreads, Cfg<D>::kDynSmem, st>>>(mq, mk, mv, offsets, order, prefix,
-                                                  static_cast<__nv_bfloat16*>(Op), lse, header, (int)T, s.H,
-                                                  s.M, s.B * s.M, s.scale * log2e, s.scale, sc);
+  kern<<<grid, kThreads, Cfg<D>::kDynSmem, st>>>(mq, mk, mv, p.grp, p.order, p.prefix,
+                                                  static_cast<__nv_bfloat16*>(p.O), p.lse, p.header, (int)p.Tq,
+                                                  p.H, p.B * p.grp.G, p.scale * log2e, p.scale, p.sc);
   MOGA_CUDA_OK(cudaGetLastError());
   return MOGA_OK;
+}
+
+moga_status launch_any(int D, const Problem& p, cudaStream_t st) {
+  return D == 128 ? launch<128>(p, st) : launch<64>(p, st);
+}
+
+// Routed groups: offsets [B, M+1] serve queries and keys alike; scratch from the workspace layout.
+Problem routed_problem(const moga_shape& s, const WsLayout& L, const void* Qp, const void* Kp, const void* Vp,
+                       const int32_t* offsets, void* O, float* lse, char* ws, const Scatter& sc) {
+  const long long T = (long long)s.N * s.k;
+  int32_t* order = reinterpret_cast<int32_t*>(ws + L.sched);
+  return Problem{s.B, s.H, T, T, s.scale, Qp, Kp, Vp, O, lse, Groups{offsets, offsets, s.M + 1, s.M},
+                 order, order + (size_t)s.B * s.M, reinterpret_cast<uint32_t*>(ws + L.header), sc};
 }
 
 }  // namespace
@@ -554,8 +598,7 @@ moga_status launch_attn_bf16(const moga_shape& s, const WsLayout& L, const void*
                              cudaStream_t st) {
   if ((long long)s.N * s.k == 0) return MOGA_OK;
   const Scatter none{nullptr, nullptr, 0, 0, 0, 0};
-  if (s.D == 128) return launch<128>(s, L, Qp, Kp, Vp, offsets, Op, lse, ws, none, st);
-  return launch<64>(s, L, Qp, Kp, Vp, offsets, Op, lse, ws, none, st);
+  return launch_any(s.D, routed_problem(s, L, Qp, Kp, Vp, offsets, Op, lse, ws, none), st);
 }
 
 moga_status launch_attn_bf16_scatter(const moga_shape& s, const WsLayout& L, const void* Qp, const void* Kp,
@@ -564,8 +607,18 @@ moga_status launch_attn_bf16_scatter(const moga_shape& s, const WsLayout& L, con
   if ((long long)s.N * s.k == 0) return MOGA_OK;
   const Strides q = qkv_strides(s);
   const Scatter sc{perm, gate, q.b, q.h, q.n, s.N};
-  if (s.D == 128) return launch<128>(s, L, Qp, Kp, Vp, offsets, O, nullptr, ws, sc, st);
-  return launch<64>(s, L, Qp, Kp, Vp, offsets, O, nullptr, ws, sc, st);
+  return launch_any(s.D, routed_problem(s, L, Qp, Kp, Vp, offsets, O, nullptr, ws, sc), st);
+}
+
+moga_status launch_attn_bf16_static(const moga_shape& s, int G, long long Tq, long long Tkv, const void* Qs,
+                                    const void* Ks, const void* Vs, const int32_t* q_offsets,
+                                    const int32_t* kv_offsets, void* Os, float* lse, char* ws, cudaStream_t st) {
+  if (Tq == 0 || G == 0) return MOGA_OK;
+  const Scatter none{nullptr, nullptr, 0, 0, 0, 0};
+  int32_t* order = reinterpret_cast<int32_t*>(ws + 256);
+  const Problem p{s.B, s.H, Tq, Tkv, s.scale, Qs, Ks, Vs, Os, lse, Groups{q_offsets, kv_offsets, 0, G},
+                  order, order + (size_t)s.B * G, reinterpret_cast<uint32_t*>(ws), none};
+  return launch_any(s.D, p, st);
 }
 
 }  // namespace moga

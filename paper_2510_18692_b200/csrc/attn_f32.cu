@@ -17,19 +17,23 @@ constexpr int kF32Keys = 32;
 template <int D>
 __global__ void __launch_bounds__(kF32Warps * 32)
 attn_f32_kernel(const float* __restrict__ Qp, const float* __restrict__ Kp,
-                const float* __restrict__ Vp, const int32_t* __restrict__ offsets,
-                float* __restrict__ Op, float* __restrict__ lse, int T, int H, int M, float scale) {
+                const float* __restrict__ Vp, const int32_t* __restrict__ q_offsets,
+                const int32_t* __restrict__ kv_offsets, int off_stride, float* __restrict__ Op,
+                float* __restrict__ lse, int Tq, int Tkv, int H, int G, float scale) {
   constexpr int KP = D + 4;  // padded K row: 16-byte reads of 8 consecutive rows are conflict-free
   __shared__ __align__(16) float Ks[kF32Keys * KP];
   __shared__ __align__(16) float Vs[kF32Keys * D];
   __shared__ int s_g, s_row0;
   const int b = blockIdx.z, h = blockIdx.y;
-  const int32_t* off = offsets + (size_t)b * (M + 1);
+  // query rows [off[g], off[g+1]) attend to key rows [koff[g], koff[g+1]); routed groups pass the
+  // same array for both, static groups (one list for all batch items) pass stride 0
+  const int32_t* off = q_offsets + (size_t)b * off_stride;
+  const int32_t* koff = kv_offsets + (size_t)b * off_stride;
   if (threadIdx.x == 0) {
     int acc = 0, found = -1, row0 = 0;
     const int rb = blockIdx.x;
-    for (int g = 0; g < M; ++g) {
-      int n = off[g + 1] - off[g];
+    for (int g = 0; g < G; ++g) {
+      int n = koff[g + 1] > koff[g] ? off[g + 1] - off[g] : 0;   // no keys: rows left untouched
       int nb = (n + kF32Warps - 1) / kF32Warps;
       if (rb < acc + nb) {
         found = g;
@@ -43,15 +47,17 @@ attn_f32_kernel(const float* __restrict__ Qp, const float* __restrict__ Kp,
   }
   __syncthreads();
   if (s_g < 0) return;
-  const int lo = off[s_g], hi = off[s_g + 1];
+  const int qlo = off[s_g], qhi = off[s_g + 1];
+  const int lo = koff[s_g], hi = koff[s_g + 1];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = s_row0 + warp;
-  const bool active = row < hi;
-  const size_t head_base = ((size_t)b * H + h) * (size_t)T;
+  const bool active = row < qhi;
+  const size_t q_base = ((size_t)b * H + h) * (size_t)Tq;
+  const size_t head_base = ((size_t)b * H + h) * (size_t)Tkv;
 
   float q[D];
   {
-    const float4* qr = reinterpret_cast<const float4*>(Qp + (head_base + (active ? row : lo)) * D);
+    const float4* qr = reinterpret_cast<const float4*>(Qp + (q_base + (active ? row : qlo)) * D);
 #pragma unroll
     for (int i = 0; i < D / 4; ++i) {
       float4 t = __ldg(qr + i);
@@ -111,26 +117,34 @@ attn_f32_kernel(const float* __restrict__ Qp, const float* __restrict__ Kp,
   if (active) {
     const float inv_l = 1.f / l;
 #pragma unroll
-    for (int i = 0; i < D / 32; ++i) Op[(head_base + row) * D + lane + 32 * i] = o[i] * inv_l;
-    if (lse != nullptr && lane == 0) lse[head_base + row] = m + logf(l);
+    for (int i = 0; i < D / 32; ++i) Op[(q_base + row) * D + lane + 32 * i] = o[i] * inv_l;
+    if (lse != nullptr && lane == 0) lse[q_base + row] = m + logf(l);
   }
 }
 
 }  // namespace
 
+moga_status launch_attn_f32_groups(int B, int H, int D, float scale, int G, int Tq, int Tkv, const float* Qp,
+                                   const float* Kp, const float* Vp, const int32_t* q_offsets,
+                                   const int32_t* kv_offsets, int off_stride, float* Op, float* lse,
+                                   cudaStream_t st) {
+  if (Tq == 0 || G == 0) return MOGA_OK;
+  dim3 grid((Tq + kF32Warps - 1) / kF32Warps + G, H, B);
+  if (D == 64)
+    attn_f32_kernel<64><<<grid, kF32Warps * 32, 0, st>>>(Qp, Kp, Vp, q_offsets, kv_offsets, off_stride, Op,
+                                                         lse, Tq, Tkv, H, G, scale);
+  else
+    attn_f32_kernel<128><<<grid, kF32Warps * 32, 0, st>>>(Qp, Kp, Vp, q_offsets, kv_offsets, off_stride, Op,
+                                                          lse, Tq, Tkv, H, G, scale);
+  MOGA_CUDA_OK(cudaGetLastError());
+  return MOGA_OK;
+}
+
 moga_status launch_attn_f32(const moga_shape& s, const float* Qp, const float* Kp, const float* Vp,
                             const int32_t* offsets, float* Op, float* lse, cudaStream_t st) {
   const int T = s.N * s.k;
-  if (T == 0) return MOGA_OK;
-  dim3 grid((T + kF32Warps - 1) / kF32Warps + s.M, s.H, s.B);
-  if (s.D == 64)
-    attn_f32_kernel<64><<<grid, kF32Warps * 32, 0, st>>>(Qp, Kp, Vp, offsets, Op, lse, T, s.H, s.M,
-                                                         s.scale);
-  else
-    attn_f32_kernel<128><<<grid, kF32Warps * 32, 0, st>>>(Qp, Kp, Vp, offsets, Op, lse, T, s.H,
-                                                          s.M, s.scale);
-  MOGA_CUDA_OK(cudaGetLastError());
-  return MOGA_OK;
+  return launch_attn_f32_groups(s.B, s.H, s.D, s.scale, s.M, T, T, Qp, Kp, Vp, offsets, offsets, s.M + 1, Op,
+                                lse, st);
 }
 
 }  // namespace moga

@@ -161,6 +161,56 @@ moga_status moga_group_attn(const moga_shape* s, const void* Qp, const void* Kp,
   return launch_attn_bf16(*s, L, Qp, Kp, Vp, offsets, Op, lse, w, cs);
 }
 
+size_t moga_static_scratch_bytes(const moga_shape* s, int32_t G) {
+  moga_status st;
+  if (!check_shape(s, &st) || G < 0) return 0;
+  return align_up(256 + sizeof(int32_t) * (2 * (size_t)s->B * G + 2), kWsAlign);
+}
+
+moga_status moga_stga_build(int32_t F, int32_t Hh, int32_t Ww, int32_t wh, int32_t ww,
+                            const int32_t* shot_starts, int32_t n_shots, int32_t tg, int32_t augment,
+                            int32_t* q_idx, int32_t* q_inv, int32_t* q_offsets, int32_t* kv_idx,
+                            int32_t* kv_offsets, int32_t* G_out, int32_t* Tkv_out) {
+  return stga_build_host(F, Hh, Ww, wh, ww, shot_starts, n_shots, tg, augment, q_idx, q_inv, q_offsets,
+                         kv_idx, kv_offsets, G_out, Tkv_out);
+}
+
+moga_status moga_gather_rows(const moga_shape* s, const int32_t* idx, int32_t L, const void* src, void* dst,
+                             void* stream) {
+  moga_status st;
+  if (!check_shape(s, &st)) return st;
+  if (L < 0 || !PTR_OK(idx) || !PTR_OK(src) || !PTR_OK(dst)) return MOGA_ERR_INVALID_ARG;
+  return launch_gather_list(*s, idx, L, src, dst, static_cast<cudaStream_t>(stream));
+}
+
+moga_status moga_static_group_attn(const moga_shape* s, int32_t G, int32_t Tq, int32_t Tkv, const void* Qs,
+                                   const void* Ks, const void* Vs, const int32_t* q_offsets,
+                                   const int32_t* kv_offsets, void* Os, float* lse, void* ws,
+                                   size_t ws_bytes, void* stream) {
+  moga_status st;
+  if (!check_shape(s, &st)) return st;
+  if (G < 0 || Tq < 0 || Tkv < 0 || !PTR_OK(Qs) || !PTR_OK(Ks) || !PTR_OK(Vs) || !PTR_OK(Os) ||
+      q_offsets == nullptr || kv_offsets == nullptr || (lse != nullptr && !aligned16(lse)))
+    return MOGA_ERR_INVALID_ARG;
+  if (!check_ws(ws, ws_bytes, moga_static_scratch_bytes(s, G), &st)) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  char* w = static_cast<char*>(ws);
+  MOGA_CUDA_OK(cudaMemsetAsync(w, 0, 256, cs));
+  if (s->dtype == MOGA_F32)
+    return launch_attn_f32_groups(s->B, s->H, s->D, s->scale, G, Tq, Tkv, static_cast<const float*>(Qs),
+                                  static_cast<const float*>(Ks), static_cast<const float*>(Vs), q_offsets,
+                                  kv_offsets, 0, static_cast<float*>(Os), lse, cs);
+  return launch_attn_bf16_static(*s, G, Tq, Tkv, Qs, Ks, Vs, q_offsets, kv_offsets, Os, lse, w, cs);
+}
+
+moga_status moga_mean3(const moga_shape* s, const void* A, const void* Bs, const int32_t* inv_b,
+                       const void* C, void* O, void* stream) {
+  moga_status st;
+  if (!check_shape(s, &st)) return st;
+  if (!PTR_OK(A) || !PTR_OK(Bs) || !PTR_OK(C) || !PTR_OK(O)) return MOGA_ERR_INVALID_ARG;
+  return launch_mean3(*s, A, Bs, inv_b, C, O, static_cast<cudaStream_t>(stream));
+}
+
 moga_status moga_unpermute(const moga_shape* s, const void* Op, const int32_t* inv,
                            const float* gate, void* O, void* stream) {
   moga_status st;

@@ -101,6 +101,23 @@ moga_status launch_attn_bf16_scatter(const moga_shape& s, const WsLayout& L, con
                                      const void* Vp, const int32_t* offsets, const int32_t* perm,
                                      const float* gate, void* O, char* ws, cudaStream_t st);
 
+// Static groups (Sec. 3.2): attention with caller-given query / key ranges per group, shared by
+// all batch items; ws holds the status header (256 B) and the schedule (2*B*G + 1 int32).
+moga_status launch_attn_bf16_static(const moga_shape& s, int G, long long Tq, long long Tkv, const void* Qs,
+                                    const void* Ks, const void* Vs, const int32_t* q_offsets,
+                                    const int32_t* kv_offsets, void* Os, float* lse, char* ws, cudaStream_t st);
+moga_status launch_attn_f32_groups(int B, int H, int D, float scale, int G, int Tq, int Tkv, const float* Qp,
+                                   const float* Kp, const float* Vp, const int32_t* q_offsets,
+                                   const int32_t* kv_offsets, int off_stride, float* Op, float* lse,
+                                   cudaStream_t st);
+moga_status launch_gather_list(const moga_shape& s, const int32_t* idx, int L, const void* src, void* dst,
+                               cudaStream_t st);
+moga_status launch_mean3(const moga_shape& s, const void* A, const void* Bs, const int32_t* inv_b, const void* C,
+                         void* O, cudaStream_t st);
+moga_status stga_build_host(int F, int Hh, int Ww, int wh, int ww, const int32_t* shot_starts, int n_shots,
+                            int tg, int augment, int32_t* q_idx, int32_t* q_inv, int32_t* q_offsets,
+                            int32_t* kv_idx, int32_t* kv_offsets, int32_t* G_out, int32_t* Tkv_out);
+
 #define MOGA_CUDA_OK(expr)                                   \
   do {                                                       \
     cudaError_t e__ = (expr);                                \
