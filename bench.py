@@ -208,8 +208,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--stage", default="all", choices=["all", "route"],
-                    help="'route' times moga_route alone on the config's X (a small resident set, for profiling)")
+    ap.add_argument("--stage", default="all", choices=["all", "route", "visual"],
+                    help="'route' times moga_route alone on the config's X (a small resident set, for profiling); "
+                         "'visual' times the whole visual-attention block: routed branch, the two static-group "
+                         "branches and their mean")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = CONFIGS[args.config]
@@ -230,6 +232,8 @@ def main():
     cfg = cfg.with_(seed=cfg.seed + 100 * rank)       # every rank works on its own layer
     if args.stage == "route":
         return run_route_only(mb, cfg, dev, args)
+    if args.stage == "visual":
+        return run_visual_block(mb, cfg, dev, args)
     inp = make_inputs(cfg, device=dev)
     sh = mb.make_shape(cfg)
     ws = mb.alloc_workspace(mb.moga_workspace_bytes(sh), dev)
@@ -364,6 +368,75 @@ def run_route_only(mb, cfg, dev, args):
     print(json.dumps({"stage": "route", "config": config_dict(cfg), "ms": ms, "GB/s": by / ms / 1e6,
                       "frac_hbm": by / ms / 1e6 / peaks["hbm_gbs"], "peak_source": peaks["source"],
                       "device_status": mb.moga_last_device_status(ws)[0]}))
+    return 0
+
+
+def run_visual_block(mb, cfg, dev, args):
+    """The visual attention block of Sec. 3.2 on the config's layer: MoGA forward, the
+    spatial-temporal static branch (4 x 4 windows, runs of 8 latent frames, synthetic shots of
+    45 latent frames, keys augmented across shot boundaries), the per-frame branch, and the mean."""
+    per_frame = 1560
+    Hh, Ww, wh, ww, tg, shot_len = 30, 52, 4, 4, 8, 45
+    if cfg.N % per_frame != 0:
+        raise SystemExit("the visual block needs a token count that is a whole number of 30x52 frames")
+    F = cfg.N // per_frame
+    inp = make_inputs(cfg, device=dev)
+    sh = mb.make_shape(cfg)
+    ws = mb.alloc_workspace(mb.moga_workspace_bytes(sh), dev)
+    lists = mb.moga_stga_build(F, Hh, Ww, wh, ww, list(range(0, F, shot_len)), tg, True)
+    G, Tkv, N = lists["G"], lists["Tkv"], cfg.N
+    d = lambda a: torch.from_numpy(a).to(dev)
+    q_idx, q_inv, kv_idx = d(lists["q_idx"]), d(lists["q_inv"]), d(lists["kv_idx"])
+    q_off, kv_off = d(lists["q_offsets"]), d(lists["kv_offsets"])
+    fr_off = torch.arange(F + 1, dtype=torch.int32, device=dev) * per_frame
+    dt = inp["Q"].dtype
+    A, C, O = (torch.empty_like(inp["Q"]) for _ in range(3))
+    Qs = torch.empty(cfg.B, cfg.H, N, cfg.D, dtype=dt, device=dev)
+    Ks, Vs = (torch.empty(cfg.B, cfg.H, Tkv, cfg.D, dtype=dt, device=dev) for _ in range(2))
+    Bs = torch.empty_like(Qs)
+    ws_st = mb.alloc_workspace(mb.moga_static_scratch_bytes(sh, G), dev)
+    ws_fr = mb.alloc_workspace(mb.moga_static_scratch_bytes(sh, F), dev)
+    names = ["moga_forward", "st_gather", "st_attn", "frame_attn", "mean3"]
+    times = {n: [] for n in names}
+    for it in range(args.warmup + args.steps):
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+        e[0].record()
+        mb.moga_forward(sh, inp["X"], inp["Wr"], inp["bias"], inp["Q"], inp["K"], inp["V"], A, ws)
+        e[1].record()
+        mb.moga_gather_rows(sh, q_idx, inp["Q"], Qs)
+        mb.moga_gather_rows(sh, kv_idx, inp["K"], Ks)
+        mb.moga_gather_rows(sh, kv_idx, inp["V"], Vs)
+        e[2].record()
+        mb.moga_static_group_attn(sh, G, N, Tkv, Qs, Ks, Vs, q_off, kv_off, Bs, None, ws_st)
+        e[3].record()
+        mb.moga_static_group_attn(sh, F, N, N, inp["Q"], inp["K"], inp["V"], fr_off, fr_off, C, None, ws_fr)
+        e[4].record()
+        mb.moga_mean3(sh, A, Bs, q_inv, C, O)
+        e[5].record()
+        torch.cuda.synchronize()
+        if it >= args.warmup:
+            for i, n in enumerate(names):
+                times[n].append(e[i].elapsed_time(e[i + 1]))
+    for w in (ws, ws_st, ws_fr):
+        code, detail = mb.moga_last_device_status(w)
+        if code != 0:
+            raise RuntimeError(f"device status {code} detail {detail:#x}")
+    ms = {n: float(np.mean(v)) for n, v in times.items()}
+    nq, nk = np.diff(lists["q_offsets"]).astype(np.float64), np.diff(lists["kv_offsets"]).astype(np.float64)
+    fl_st = cfg.B * cfg.H * 4.0 * cfg.D * float((nq * nk).sum())
+    fl_fr = cfg.B * cfg.H * 4.0 * cfg.D * F * float(per_frame) ** 2
+    es = 2 if cfg.dtype == "bf16" else 4
+    row = cfg.B * cfg.H * cfg.D * es
+    peaks = load_peaks()
+    print(json.dumps({
+        "stage": "visual", "config": config_dict(cfg),
+        "static_groups": {"frames": F, "windows": [wh, ww], "run_frames": tg, "shot_frames": shot_len, "groups": G,
+                          "queries_per_group": [int(nq.min()), int(nq.max())], "keys_per_group": [int(nk.min()), int(nk.max())]},
+        "ms": ms, "ms_total": sum(ms.values()),
+        "st_attn_TFLOP/s": fl_st / ms["st_attn"] / 1e9, "frame_attn_TFLOP/s": fl_fr / ms["frame_attn"] / 1e9,
+        "st_gather_GB/s": 2.0 * row * (N + 2 * Tkv) / ms["st_gather"] / 1e6,
+        "mean3_GB/s": 4.0 * row * N / ms["mean3"] / 1e6, "hbm_peak_GB/s": peaks["hbm_gbs"],
+        "useful_tflop": {"st": fl_st / 1e12, "frame": fl_fr / 1e12}}))
     return 0
 
 
