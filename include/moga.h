@@ -247,6 +247,28 @@ moga_status moga_forward(const moga_shape* s, const void* X, const float* Wr, co
                          size_t ws_bytes, void* stream);
 
 /*
+ * The whole forward from HOST buffers (the call for a caller whose activations live in host
+ * memory).  X, Wr, bias, Q, K, V, O, gid_out, gate_out are HOST pointers (page-locked memory
+ * is needed for the copies to overlap; pageable memory works but serialises); Q, K, V, O are
+ * contiguous [B, H, N, D] (strides in the shape must be zero).  `arena` is device memory of
+ * at least moga_forward_host_bytes(s, heads_per_chunk), 256-byte aligned: it holds X, the
+ * routing results, two staging sets of heads_per_chunk heads of Q/K/V and of O, and one
+ * permuted chunk.  One internal stream copies X and then Q/K/V chunk by chunk, `stream`
+ * routes, sorts and runs gather + group attention (+ gated inverse permutation) on each
+ * chunk as its inputs land, a second internal stream returns each chunk of O; `stream`
+ * finally waits for the last copy, so synchronising it means O is on the host.  Results are
+ * bit-identical to moga_forward.  The two streams and a fixed pool of events are created on
+ * the first call on each device (no memory is allocated); calls on one device must not
+ * overlap (they share those events).  At most 64 chunks.  The device status word is at the
+ * start of `arena` (moga_last_device_status(arena, ...)).
+ */
+size_t moga_forward_host_bytes(const moga_shape* s, int32_t heads_per_chunk);
+moga_status moga_forward_host(const moga_shape* s, const void* X, const float* Wr, const float* bias,
+                              const void* Q, const void* K, const void* V, void* O, int32_t* gid_out,
+                              float* gate_out, void* arena, size_t arena_bytes, int32_t heads_per_chunk,
+                              void* stream);
+
+/*
  * Synchronises `stream`, reads the device status word kept at the start of ws and
  * clears it.  Every permute / group_attn / forward call resets the word when it
  * starts, so the result describes the most recent such call on this ws: MOGA_OK,

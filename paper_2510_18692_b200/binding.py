@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libmoga.so")
 EXPORTS = ("moga_workspace_bytes", "moga_scratch_bytes", "moga_status_string", "moga_route",
            "moga_permute", "moga_group_attn", "moga_unpermute", "moga_forward",
            "moga_last_device_status", "moga_sort_static", "moga_balance_stats", "moga_stga_build", "moga_gather_rows",
-           "moga_static_group_attn", "moga_mean3")
+           "moga_static_group_attn", "moga_mean3", "moga_forward_host_bytes", "moga_forward_host")
 
 MOGA_F32, MOGA_BF16 = 0, 1
 MOGA_ROUTE_AUTO, MOGA_ROUTE_ALU = 0, 1
@@ -48,12 +48,11 @@ if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2510_18692_b200.build` "
                       "(there is no CPU fallback)")
 lib = ctypes.CDLL(LIB_PATH)
-lib.moga_workspace_bytes.restype = ctypes.c_size_t
-lib.moga_scratch_bytes.restype = ctypes.c_size_t
-lib.moga_static_scratch_bytes.restype = ctypes.c_size_t
-lib.moga_status_string.restype = ctypes.c_char_p
-for _n in EXPORTS[3:]:
+for _n in EXPORTS:
     getattr(lib, _n).restype = ctypes.c_int
+for _n in ("moga_workspace_bytes", "moga_scratch_bytes", "moga_static_scratch_bytes", "moga_forward_host_bytes"):
+    getattr(lib, _n).restype = ctypes.c_size_t
+lib.moga_status_string.restype = ctypes.c_char_p
 
 
 def status_string(code: int) -> str:
@@ -176,6 +175,18 @@ def moga_forward(shape, X, Wr, bias, Q, K, V, O, ws, gid_out=None, gate_out=None
                             _ptr(V), _ptr(O), _ptr(gid_out), _ptr(gate_out), _ptr(perm_out),
                             _ptr(offsets_out), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()),
            "moga_forward")
+
+
+def moga_forward_host_bytes(shape, heads_per_chunk) -> int:
+    return int(lib.moga_forward_host_bytes(ctypes.byref(shape), ctypes.c_int32(heads_per_chunk)))
+
+
+def moga_forward_host(shape, X, Wr, bias, Q, K, V, O, arena, heads_per_chunk, gid_out=None, gate_out=None):
+    """Forward from host tensors (torch CPU tensors, ideally pinned); ``arena`` is a CUDA uint8 tensor."""
+    _check(lib.moga_forward_host(ctypes.byref(shape), _ptr(X), _ptr(Wr), _ptr(bias), _ptr(Q), _ptr(K), _ptr(V),
+                                 _ptr(O), _ptr(gid_out), _ptr(gate_out), _ptr(arena),
+                                 ctypes.c_size_t(arena.numel()), ctypes.c_int32(heads_per_chunk), _stream()),
+           "moga_forward_host")
 
 
 def moga_last_device_status(ws):
