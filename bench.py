@@ -208,6 +208,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--sharding", default="layers", choices=["layers", "heads"],
+                    help="with --gpus N > 1: 'layers' gives every rank its own layer (weak scaling, no collective); "
+                         "'heads' splits ONE layer: tokens of X for routing, heads of Q/K/V for attention, with the "
+                         "all-gather of the routing results as the only exchange (strong scaling)")
     ap.add_argument("--stage", default="all", choices=["all", "route", "visual"],
                     help="'route' times moga_route alone on the config's X (a small resident set, for profiling); "
                          "'visual' times the whole visual-attention block: routed branch, the two static-group "
@@ -230,6 +234,8 @@ def main():
     from paper_2510_18692_b200 import binding as mb   # raises if the CUDA library is missing
 
     cfg = cfg.with_(seed=cfg.seed + 100 * rank)       # every rank works on its own layer
+    if args.sharding == "heads":
+        return run_head_sharded(mb, CONFIGS[args.config], dev, args, rank, world)
     if args.stage == "route":
         return run_route_only(mb, cfg, dev, args)
     if args.stage == "visual":
@@ -368,6 +374,49 @@ def run_route_only(mb, cfg, dev, args):
     print(json.dumps({"stage": "route", "config": config_dict(cfg), "ms": ms, "GB/s": by / ms / 1e6,
                       "frac_hbm": by / ms / 1e6 / peaks["hbm_gbs"], "peak_source": peaks["source"],
                       "device_status": mb.moga_last_device_status(ws)[0]}))
+    return 0
+
+
+def run_head_sharded(mb, cfg, dev, args, rank, world):
+    """One layer split over the ranks (strong scaling): see paper_2510_18692_b200/sharded.py."""
+    from paper_2510_18692_b200.sharded import forward_head_sharded, shard_bounds
+    lo, hi = shard_bounds(cfg.N, world, rank)
+    h_lo, h_hi = shard_bounds(cfg.H, world, rank)
+    inp = make_inputs(cfg, device=dev, heads=list(range(h_lo, h_hi)))      # every rank draws the same layer
+    X_local = inp["X"][:, lo:hi].contiguous()
+    del inp["X"]
+    O = torch.empty_like(inp["Q"])
+
+    def step():
+        return forward_head_sharded(mb, cfg, X_local, inp["Wr"], inp["bias"], inp["Q"], inp["K"], inp["V"], O)
+
+    for _ in range(args.warmup):
+        _, _, offsets = step()
+    sizes = np.diff(offsets.cpu().numpy(), axis=1)
+    flops_local = sum(useful_flops(sizes[b], h_hi - h_lo, cfg.D) for b in range(cfg.B))
+    clocks = ClockSampler(dev.index or 0)
+    clocks.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    barrier_sync()
+    ev[0].record()
+    for _ in range(args.steps):
+        step()
+    ev[1].record()
+    barrier_sync()
+    clk = clocks.stop()
+    ms, total_flops = aggregate(ev[0].elapsed_time(ev[1]) / args.steps, flops_local, dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": total_flops / (ms * 1e-3) / 1e12, "unit": "TFLOP/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+            "config": dict(config_dict(cfg), sharding="tokens for routing, heads for attention; one all-gather of (gid, gate)"),
+            "gpu_launches": (kernels_per_forward(cfg) + (1 if cfg.k == 1 and cfg.dtype == "bf16" else 0)) * args.steps,
+            "clocks": clk}))
     return 0
 
 

@@ -1,0 +1,67 @@
+"""Sharding semantics of the multi-GPU path checked on one GPU, rank by rank and without any
+collective: routing token shards separately gives the bits of routing the whole sequence,
+and running the stages on head shards gives the bits of running them on all heads."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from parity import check_output, to_np32
+from paper_2510_18692_b200.inputs import GATE_SOFTMAX_TOPK, MogaConfig, make_inputs
+from paper_2510_18692_b200.sharded import forward_head_sharded, shard_bounds
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mb():
+    from paper_2510_18692_b200 import build
+    build.build()
+    from paper_2510_18692_b200 import binding
+    return binding
+
+
+def test_shards_reproduce_the_unsharded_stages(mb):
+    cfg = MogaConfig("sh", 2, 5, 1777, 256, 128, 8, 2, "bf16", GATE_SOFTMAX_TOPK, 41)
+    inp = make_inputs(cfg, device="cuda")
+    # world size 1: the sharded driver is the staged forward
+    O = torch.empty_like(inp["Q"])
+    gid, gate, offsets = forward_head_sharded(mb, cfg, inp["X"], inp["Wr"], inp["bias"], inp["Q"], inp["K"],
+                                              inp["V"], O)
+    torch.cuda.synchronize()
+    host = {k: to_np32(v) for k, v in inp.items()}
+    off, perm, _ = oracle.sort(gid.cpu().numpy(), cfg.M)
+    want = oracle.attn_all(host["Q"], host["K"], host["V"], gid.cpu().numpy(), gate.double().cpu().numpy(), off,
+                           perm, cfg.scale)
+    check_output(O.float().cpu().numpy(), want, "bf16")
+    world = 3
+    # routing token shards one by one (what each rank would do) and concatenating
+    parts_g, parts_t = [], []
+    for r in range(world):
+        lo, hi = shard_bounds(cfg.N, world, r)
+        sh = mb.make_shape(cfg.with_(N=hi - lo))
+        g = torch.empty(cfg.B, hi - lo, cfg.k, dtype=torch.int32, device="cuda")
+        t = torch.empty(cfg.B, hi - lo, cfg.k, dtype=torch.float32, device="cuda")
+        ws = mb.alloc_workspace(mb.moga_scratch_bytes(sh))
+        mb.moga_route(sh, inp["X"][:, lo:hi].contiguous(), inp["Wr"], inp["bias"], g, t, None, ws)
+        parts_g.append(g)
+        parts_t.append(t)
+    assert torch.equal(torch.cat(parts_g, 1), gid) and torch.equal(torch.cat(parts_t, 1), gate)
+    # head shards one by one with the gathered routing
+    T = cfg.N * cfg.k
+    for r in range(world):
+        lo, hi = shard_bounds(cfg.H, world, r)
+        cfg_h = cfg.with_(H=hi - lo)
+        sh = mb.make_shape(cfg_h)
+        ws = mb.alloc_workspace(mb.moga_scratch_bytes(sh))
+        perm_d = torch.empty(cfg.B, T, dtype=torch.int32, device="cuda")
+        inv = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.int32, device="cuda")
+        offs = torch.empty(cfg.B, cfg.M + 1, dtype=torch.int32, device="cuda")
+        Qh, Kh, Vh = (inp[n][:, lo:hi].contiguous() for n in ("Q", "K", "V"))
+        Qp, Kp, Vp, Op = (torch.empty(cfg.B, hi - lo, T, cfg.D, dtype=torch.bfloat16, device="cuda") for _ in range(4))
+        Oh = torch.empty_like(Qh)
+        mb.moga_permute(sh, gid, Qh, Kh, Vh, perm_d, inv, offs, Qp, Kp, Vp, ws)
+        mb.moga_group_attn(sh, Qp, Kp, Vp, offs, Op, None, ws)
+        mb.moga_unpermute(sh, Op, inv, gate, Oh)
+        torch.cuda.synchronize()
+        assert torch.equal(offs, offsets) and torch.equal(Oh, O[:, lo:hi])
