@@ -2,6 +2,7 @@
 itself -- a library routine (numpy matmul / argsort, torch SDPA), a pure-Python
 brute force that never sorts, a closed form, or an invariant the paper fixes."""
 import math
+import os
 
 import numpy as np
 import pytest
@@ -360,3 +361,24 @@ def test_static_group_attention_special_cases():
     O3 = oracle.static_group_attn(Q, K3, V, qg, kg, scale)
     assert np.abs(O1[:, :, shot1] - O3[:, :, shot1]).max() > 1e-4
     assert np.abs(oracle.mean3(O1, O2, O3) - (O1 + O2 + O3) / 3).max() == 0
+
+
+# ----------------------------------------------------------------------------- printed sparsity (Table 4)
+def test_group_sizes_reproduce_the_printed_sparsity_steps():
+    """Under uniform assignment the routed branch computes 1/M of the query-key pairs
+    (Sec. 3.2, complexity paragraph).  The paper's sparsity column also contains the static
+    branches, a constant density, so the DIFFERENCE between two rows is free of it:
+    sparsity(M2) - sparsity(M1) = 1/M1 - 1/M2.  The pair count comes from the oracle's sort of
+    a balanced assignment (sum of squared group sizes), the numbers from the printed table."""
+    path = os.path.join(os.path.dirname(__file__), "golden", "table4_sparsity.txt")
+    rows = [tuple(map(float, l.split())) for l in open(path) if l.strip() and not l.startswith("#")]
+    N = 2 * 4 * 5 * 8 * 3
+    density = {}
+    for M, _ in rows:
+        M = int(M)
+        gid = (np.arange(N) % M).astype(np.int32).reshape(1, N, 1)
+        offsets, _, _ = oracle.sort(gid, M)
+        density[M] = float((np.diff(offsets[0]).astype(np.float64) ** 2).sum()) / N ** 2
+        assert abs(density[M] - 1.0 / M) < 1e-15
+    for (M1, s1), (M2, s2) in zip(rows, rows[1:]):
+        assert abs((s2 - s1) / 100.0 - (density[int(M1)] - density[int(M2)])) < 1e-12
