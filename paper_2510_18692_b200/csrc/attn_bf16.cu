@@ -13,8 +13,10 @@
 //               Online softmax in the log2 domain against a reference maximum taken
 //               from the row's first tile; it is raised, and O rescaled in TMEM by
 //               the same warps, only when a later tile's row sum exceeds 2^40.
-//               They also run the epilogue:
-//               O / l -> bf16 -> shared memory -> coalesced, row-predicated stores.
+//               They also run the epilogue: O / l -> bf16 -> a 2 KB staging buffer
+//               private to the warp -> 64-byte row segments, row-predicated stores.
+//               (The Q tiles are released by the MMA warp right after their last
+//               use, so the next item's Q loads overlap this item's tail.)
 //
 // TMEM (512 columns): S_A [0,128) S_B [128,256) O_A [256,256+D) O_B [384,384+D);
 // P (bf16, two per column) overwrites the first 64 columns of its S tile.
@@ -127,8 +129,9 @@ struct Cfg {
   static constexpr int kSmemQ = 0;
   static constexpr int kSmemK = 2 * kTileBytes;
   static constexpr int kSmemV = kSmemK + NS * kTileBytes;
-  static constexpr int kSmemBar = kSmemV + NS * kTileBytes;
-  static constexpr int kNumBars = 2 + 2 + 4 * NS + 2 + 2 + 2 + 2 + 2;
+  static constexpr int kSmemStage = kSmemV + NS * kTileBytes;   // 8 softmax warps x 2 KB output staging
+  static constexpr int kSmemBar = kSmemStage + 8 * 2048;
+  static constexpr int kNumBars = 2 + 2 + 4 * NS + 2 + 2 + 2 + 2;
   static constexpr int kSmemTotal = kSmemBar + 8 * kNumBars + 16;
   static constexpr int kDynSmem = kSmemTotal + 1024;      // slack for 1024-byte alignment
 };
@@ -165,7 +168,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
   const uint32_t bars = base + C::kSmemBar;
   constexpr int Q_FULL = 0, Q_EMPTY = 2, K_FULL = 4, K_EMPTY = 4 + NS, V_FULL = 4 + 2 * NS,
                 V_EMPTY = 4 + 3 * NS, S_FULL = 4 + 4 * NS, P_FULL = S_FULL + 2, O_FULL = S_FULL + 4,
-                O_EMPTY = S_FULL + 6, STG_FULL = S_FULL + 8;
+                O_EMPTY = S_FULL + 6;
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + C::kSmemBar + 8 * C::kNumBars);
   volatile uint32_t* abort_flag = tmem_slot + 1;
@@ -176,12 +179,11 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar(Q_FULL + i), 1);
-      mbar_init(bar(Q_EMPTY + i), kTileM);
+      mbar_init(bar(Q_EMPTY + i), 1);
       mbar_init(bar(S_FULL + i), 1);
       mbar_init(bar(P_FULL + i), kTileM);
       mbar_init(bar(O_FULL + i), 1);
       mbar_init(bar(O_EMPTY + i), kTileM);
-      mbar_init(bar(STG_FULL + i), kTileM);
     }
     for (int i = 0; i < NS; ++i) {
       mbar_init(bar(K_FULL + i), 1);
@@ -311,6 +313,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         for (int x = 0; x < nx; ++x) {
           issue_qk(x, nk % NS);
           tc_commit(bar(S_FULL + x));
+          if (ntiles == 1) tc_commit(bar(Q_EMPTY + x));   // the item's only use of this Q tile
         }
         tc_commit(bar(K_EMPTY + nk % NS));
         ++nk;
@@ -336,6 +339,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             if (more) {
               issue_qk(x, nk % NS);
               tc_commit(bar(S_FULL + x));
+              if (j + 2 == ntiles) tc_commit(bar(Q_EMPTY + x));   // last use of this Q tile: free it early
             } else {
               tc_commit(bar(O_FULL + x));
             }
@@ -361,7 +365,6 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     const uint32_t tS = tmem + lane_off + x * kTileN;
     const uint32_t tO = tmem + lane_off + 256 + x * 128;
-    unsigned char* stage = smem + C::kSmemQ + x * C::kTileBytes;    // O staging reuses the Q tile
     uint32_t n_s = 0, n_o = 0;
     bool ok = true;
     for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
@@ -444,21 +447,40 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         mbar_arrive(bar(P_FULL + x));
       }
       if (!ok) break;
-      // ---- epilogue: O / l -> bf16 -> shared -> global
+      // ---- epilogue: O / l -> bf16 -> per-warp staging -> global
       ok = wait(O_FULL + x, n_o & 1u, 11);
       if (!ok) break;
       ++n_o;
       tc_fence_after();
       float inv_l = 1.f / l;
-      if (sc.perm != nullptr && tile_row0 + r < it.qhi) {
-        const int b = it.bh / H;
-        inv_l *= sc.gate[(size_t)b * sc.N + sc.perm[(size_t)b * T + tile_row0 + r]];
+      const bool live = tile_row0 + r < it.qhi;
+      const int bb = it.bh / H, hh = it.bh % H;
+      if (sc.perm != nullptr && live) inv_l *= sc.gate[(size_t)bb * sc.N + sc.perm[(size_t)bb * T + tile_row0 + r]];
+      // Each warp stages 32 rows x 32 columns (2 KB) at a time in its own buffer and writes them
+      // out itself: lane L stores piece L % 4 of rows i * 8 + L / 4, i = 0..3 (64-byte row segments).
+      unsigned char* wst = smem + C::kSmemStage + (x * 4 + q) * 2048;
+      __nv_bfloat16* obase[4];
+      bool orow_live[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int grow = tile_row0 + q * 32 + i * 8 + (lane >> 2);
+        orow_live[i] = grow < it.qhi;
+        if (sc.perm != nullptr) {
+          const int tok = orow_live[i] ? sc.perm[(size_t)bb * T + grow] : 0;
+          obase[i] = Op + bb * sc.sb + hh * sc.sh + (long long)tok * sc.sn;
+        } else {
+          obase[i] = Op + ((size_t)it.bh * T + grow) * D;
+        }
       }
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
         uint32_t oreg[32];
         tmem_ld32(tO + c * 32, oreg);
         tmem_wait_ld();
+        if (c == D / 32 - 1) {
+          tc_fence_before();
+          mbar_arrive(bar(O_EMPTY + x));    // TMEM O (and S) of this tile may be overwritten
+        }
 #pragma unroll
         for (int v = 0; v < 4; ++v) {      // four 16-byte chunks (8 bf16 each) per 32 columns
           uint4 pk;
@@ -469,43 +491,18 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                                                      __uint_as_float(oreg[v * 8 + 2 * i + 1]) * inv_l);
             pw[i] = *reinterpret_cast<uint32_t*>(&t);
           }
-          const int chunk = c * 4 + v;     // 16-byte chunk index inside the row
-          *reinterpret_cast<uint4*>(stage + r * (D * 2) + ((chunk ^ (r & 7)) * 16)) = pk;
+          *reinterpret_cast<uint4*>(wst + lane * 64 + ((v ^ ((lane >> 1) & 3)) * 16)) = pk;
         }
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int row = i * 8 + (lane >> 2), piece = lane & 3;
+          const uint4 val = *reinterpret_cast<const uint4*>(wst + row * 64 + ((piece ^ ((row >> 1) & 3)) * 16));
+          if (orow_live[i]) *reinterpret_cast<uint4*>(obase[i] + c * 32 + piece * 8) = val;
+        }
+        __syncwarp();
       }
-      tc_fence_before();
-      mbar_arrive(bar(O_EMPTY + x));        // TMEM O (and S) of this tile may be overwritten
-      if (lse != nullptr && tile_row0 + r < it.qhi)
-        lse[(size_t)it.bh * T + tile_row0 + r] = m * scale + __logf(l);
-      mbar_arrive(bar(STG_FULL + x));          // all 128 rows staged (bounded wait, no bar.sync)
-      ok = wait(STG_FULL + x, (n_o & 1u) ^ 1u, 12);
-      if (!ok) break;
-      constexpr int kChunks = D * 2 / 16;   // 16-byte chunks per row
-      const int t = threadIdx.x - (4 + 4 * x) * 32;
-      if (sc.perm == nullptr) {
-#pragma unroll 4
-        for (int id = t; id < kTileM * kChunks; id += kTileM) {
-          const int row = id / kChunks, chunk = id % kChunks;
-          if (tile_row0 + row < it.qhi) {
-            const uint4 val = *reinterpret_cast<const uint4*>(stage + row * (D * 2) + ((chunk ^ (row & 7)) * 16));
-            *reinterpret_cast<uint4*>(Op + ((size_t)it.bh * T + tile_row0 + row) * D + chunk * 8) = val;
-          }
-        }
-      } else {
-        const int b = it.bh / H, h = it.bh % H;
-        __nv_bfloat16* obase = Op + b * sc.sb + h * sc.sh;
-        const int32_t* prow = sc.perm + (size_t)b * T + tile_row0;
-#pragma unroll 4
-        for (int id = t; id < kTileM * kChunks; id += kTileM) {
-          const int row = id / kChunks, chunk = id % kChunks;
-          if (tile_row0 + row < it.qhi) {
-            const uint4 val = *reinterpret_cast<const uint4*>(stage + row * (D * 2) + ((chunk ^ (row & 7)) * 16));
-            *reinterpret_cast<uint4*>(obase + (long long)prow[row] * sc.sn + chunk * 8) = val;
-          }
-        }
-      }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_arrive(bar(Q_EMPTY + x));        // the producer may load the next Q tile here
+      if (lse != nullptr && live) lse[(size_t)it.bh * T + tile_row0 + r] = m * scale + __logf(l);
     }
   }
 
