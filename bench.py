@@ -152,8 +152,10 @@ def oracle_sample(cfg, host, routing, target_s=12.0):
         oracle.attn_rows(host["Q"], host["K"], host["V"], gid, gate, offsets, perm, cfg.scale, rows)
         return time.perf_counter() - t0, fl
 
-    t_cal, fl_cal = run(64, 1)
-    nrows = int(max(64, min(200000, 64 * target_s / max(t_cal, 1e-4))))
+    t_cal, _ = run(64, 1)                    # includes thread start-up: only good for a first guess
+    n2 = int(max(64, min(50000, 64 * 2.0 / max(t_cal, 1e-4))))
+    t2, _ = run(n2, 3)                       # a ~2 s run calibrates the real one
+    nrows = int(max(64, min(400000, n2 * target_s / max(t2, 1e-4))))
     t, fl = run(nrows, 2)
     return dict(tflops=fl / t / 1e12, seconds=t, rows=nrows, flops=fl, route_tokens=len(tok),
                 route_seconds=t_route, cores=oracle.threads())
