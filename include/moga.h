@@ -31,6 +31,8 @@
  *      offsets [B, M+1]         int32          group g owns positions [offsets[g], offsets[g+1])
  *      Qp,Kp,Vp,Op [B, H, T, D] dtype          rows in sorted (group-major) order, contiguous
  *      lse     [B, H, T]        float          optional log-sum-exp of the scaled scores
+ *  - N = 0 (no tokens) is valid: the stage and forward calls return MOGA_OK without reading the
+ *    data pointers; moga_permute / moga_forward still zero the offsets they are given.
  *  - Limits: 1 <= M <= 64, 1 <= k <= min(M, 8), D in {64, 128}, C a multiple of
  *    16 bytes worth of elements, N*k < 2^31.  Outside them: MOGA_ERR_UNSUPPORTED.
  */

@@ -93,6 +93,7 @@ moga_status moga_route(const moga_shape* s, const void* X, const float* Wr, cons
                        void* stream) {
   moga_status st;
   if (!check_shape(s, &st)) return st;
+  if (s->N == 0) return MOGA_OK;                  // no tokens: nothing to write
   if (!PTR_OK(X) || !PTR_OK(Wr) || !PTR_OK(gid) || !PTR_OK(gate) ||
       (bias != nullptr && !aligned16(bias)) || (logits != nullptr && !aligned16(logits)))
     return MOGA_ERR_INVALID_ARG;
@@ -126,6 +127,11 @@ moga_status moga_permute(const moga_shape* s, const int32_t* gid, const void* Q,
                          void* Kp, void* Vp, void* ws, size_t ws_bytes, void* stream) {
   moga_status st;
   if (!check_shape(s, &st)) return st;
+  if (s->N == 0) {                                // no tokens: every group is empty
+    if (!PTR_OK(offsets)) return MOGA_ERR_INVALID_ARG;
+    MOGA_CUDA_OK(cudaMemsetAsync(offsets, 0, sizeof(int32_t) * s->B * (s->M + 1), static_cast<cudaStream_t>(stream)));
+    return MOGA_OK;
+  }
   if (!PTR_OK(gid) || !PTR_OK(perm) || !PTR_OK(inv) || !PTR_OK(offsets)) return MOGA_ERR_INVALID_ARG;
   const int n_out = (Qp != nullptr) + (Kp != nullptr) + (Vp != nullptr);
   if (n_out != 0 && n_out != 3) return MOGA_ERR_INVALID_ARG;
@@ -147,6 +153,7 @@ moga_status moga_group_attn(const moga_shape* s, const void* Qp, const void* Kp,
                             size_t ws_bytes, void* stream) {
   moga_status st;
   if (!check_shape(s, &st)) return st;
+  if (s->N == 0) return MOGA_OK;
   if (!PTR_OK(Qp) || !PTR_OK(Kp) || !PTR_OK(Vp) || !PTR_OK(offsets) || !PTR_OK(Op) ||
       (lse != nullptr && !aligned16(lse)))
     return MOGA_ERR_INVALID_ARG;
@@ -215,6 +222,7 @@ moga_status moga_unpermute(const moga_shape* s, const void* Op, const int32_t* i
                            const float* gate, void* O, void* stream) {
   moga_status st;
   if (!check_shape(s, &st)) return st;
+  if (s->N == 0) return MOGA_OK;
   if (!PTR_OK(Op) || !PTR_OK(inv) || !PTR_OK(gate) || !PTR_OK(O)) return MOGA_ERR_INVALID_ARG;
   return launch_unpermute(*s, Op, inv, gate, O, static_cast<cudaStream_t>(stream));
 }
@@ -225,6 +233,11 @@ moga_status moga_forward(const moga_shape* s, const void* X, const float* Wr, co
                          size_t ws_bytes, void* stream) {
   moga_status st;
   if (!check_shape(s, &st)) return st;
+  if (s->N == 0) {                                // no tokens: only the (all-zero) offsets exist
+    if (offsets_out)
+      MOGA_CUDA_OK(cudaMemsetAsync(offsets_out, 0, sizeof(int32_t) * s->B * (s->M + 1), static_cast<cudaStream_t>(stream)));
+    return MOGA_OK;
+  }
   if (!PTR_OK(X) || !PTR_OK(Wr) || !PTR_OK(Q) || !PTR_OK(K) || !PTR_OK(V) || !PTR_OK(O) ||
       (bias != nullptr && !aligned16(bias)))
     return MOGA_ERR_INVALID_ARG;

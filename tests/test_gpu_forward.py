@@ -174,3 +174,25 @@ def test_multishot_bf16_full_size_sampled(mb):
 
 def test_skew_bf16_full_size_sampled(mb):
     sampled_parity(mb, CONFIGS["skew_bf16"], n_rows=768)
+
+
+def test_single_token_and_no_token(mb):
+    """N = 1: the token attends to itself, so O = gate * V.  N = 0: nothing is read or written
+    but the offsets, which are all zero."""
+    cfg = MogaConfig("one", 2, 3, 1, 64, 128, 4, 1, "bf16", GATE_SOFTMAX_ALL, 17)
+    inp = make_inputs(cfg, device="cuda")
+    O, gid, gate, perm, offsets = run_forward(mb, cfg, inp)
+    want = (inp["V"].float() * gate[:, None, :, :]).bfloat16()
+    assert torch.equal(O, want)
+    assert torch.all(perm == 0) and int(offsets[:, -1].sum()) == 2
+    empty = cfg.with_(N=0)
+    sh = mb.make_shape(empty)
+    ws = mb.alloc_workspace(max(mb.moga_workspace_bytes(sh), 256))
+    off = torch.full((2, 5), 9, dtype=torch.int32, device="cuda")
+    mb.moga_forward(sh, None, None, None, None, None, None, None, ws, None, None, None, off)
+    mb.moga_permute(sh, None, None, None, None, None, None, off, None, None, None, ws)
+    mb.moga_route(sh, None, None, None, None, None)
+    mb.moga_group_attn(sh, None, None, None, None, None, None, ws)
+    mb.moga_unpermute(sh, None, None, None, None)
+    torch.cuda.synchronize()
+    assert torch.all(off == 0)
