@@ -144,3 +144,64 @@ def test_visual_attention_block(mb, dtype):
     ref = (A.double() + Bt.double() + C.double()) / 3
     tol = 2.0 ** -8 * ref.abs().max().item() if dtype == "bf16" else 1e-6
     assert (O.double() - ref).abs().max().item() <= tol
+
+
+def _static_rows_oracle(Q, K, V, q_groups, kv_groups, scale, rows):
+    """fp64 rows of the static group attention, one (b, h, token) at a time, from the definition."""
+    owner = {}
+    for g, qi in enumerate(q_groups):
+        for n in qi:
+            owner[int(n)] = g
+    out = np.empty((len(rows), Q.shape[-1]))
+    for i, (b, h, n) in enumerate(rows):
+        ki = kv_groups[owner[int(n)]]
+        s = (K[b, h, ki].astype(np.float64) @ Q[b, h, n].astype(np.float64)) * scale
+        p = np.exp(s - s.max())
+        out[i] = (p / p.sum()) @ V[b, h, ki].astype(np.float64)
+    return out
+
+
+@pytest.mark.parametrize("name", ["clip_bf16", "minute_bf16"])
+def test_static_branches_full_size_sampled(mb, name):
+    """The static branches in the configuration bench.py --stage visual times (4 x 4 windows, runs of
+    8 latent frames, shots of 45 latent frames) at paper sizes, checked on sampled rows: first and
+    last query of a sample of groups (shot-boundary groups included) and random tokens."""
+    from paper_2510_18692_b200.inputs import CONFIGS
+    cfg = CONFIGS[name]
+    free, _ = torch.cuda.mem_get_info()
+    es = 2
+    if free < 9 * cfg.B * cfg.H * cfg.N * cfg.D * es + cfg.B * cfg.N * cfg.C * es + (2 << 30):
+        pytest.skip("not enough device memory for this size")
+    Hh, Ww, wh, ww, tg, shot_len = 30, 52, 4, 4, 8, 45
+    F = cfg.N // (Hh * Ww)
+    shots = list(range(0, F, shot_len))
+    inp = make_inputs(cfg, device="cuda")
+    del inp["X"]
+    lists = mb.moga_stga_build(F, Hh, Ww, wh, ww, shots, tg, True)
+    Bs, _ = run_static(mb, cfg, inp["Q"], inp["K"], inp["V"], lists["q_idx"], lists["kv_idx"],
+                       lists["q_offsets"], lists["kv_offsets"])
+    sh = mb.make_shape(cfg)
+    fr_off = (np.arange(F + 1) * Hh * Ww).astype(np.int32)
+    C = torch.empty_like(inp["Q"])
+    ws = mb.alloc_workspace(mb.moga_static_scratch_bytes(sh, F))
+    mb.moga_static_group_attn(sh, F, cfg.N, cfg.N, inp["Q"], inp["K"], inp["V"], _dev(fr_off), _dev(fr_off), C, None, ws)
+    assert mb.moga_last_device_status(ws) == (0, 0)
+    qg, kg = oracle.stga_groups(F, Hh, Ww, wh, ww, shots, tg)
+    assert len(qg) == lists["G"]
+    rng = np.random.default_rng(5)
+    heads = [0, cfg.H - 1]
+    pick = sorted(set(rng.choice(len(qg), size=min(24, len(qg)), replace=False).tolist()) | {0, len(qg) - 1} |
+                  {g for g in range(len(qg)) if len(kg[g]) > len(qg[g])} & set(range(0, len(qg), 7)))
+    toks = [int(qg[g][0]) for g in pick] + [int(qg[g][-1]) for g in pick] + rng.integers(0, cfg.N, 64).tolist()
+    rows = [(0, h, n) for n in toks for h in heads]
+    Qh, Kh, Vh = (to_np32(inp[n][:, heads]) for n in ("Q", "K", "V"))
+    rows_h = [(b, heads.index(h), n) for b, h, n in rows]
+    want_st = _static_rows_oracle(Qh, Kh, Vh, qg, kg, cfg.scale, rows_h)
+    fq, fk = oracle.frame_groups(F, Hh, Ww)
+    want_fr = _static_rows_oracle(Qh, Kh, Vh, fq, fk, cfg.scale, rows_h)
+    q_inv = torch.from_numpy(lists["q_inv"].astype(np.int64)).cuda()
+    bi = torch.tensor([r[0] for r in rows]).cuda()
+    hi = torch.tensor([r[1] for r in rows]).cuda()
+    ni = torch.tensor([r[2] for r in rows]).cuda()
+    check_output(Bs[bi, hi, q_inv[ni]].float().cpu().numpy(), want_st, "bf16", "spatial-temporal rows")
+    check_output(C[bi, hi, ni].float().cpu().numpy(), want_fr, "bf16", "per-frame rows")

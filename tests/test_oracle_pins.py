@@ -382,3 +382,19 @@ def test_group_sizes_reproduce_the_printed_sparsity_steps():
         assert abs(density[M] - 1.0 / M) < 1e-15
     for (M1, s1), (M2, s2) in zip(rows, rows[1:]):
         assert abs((s2 - s1) / 100.0 - (density[int(M1)] - density[int(M2)])) < 1e-12
+
+
+def test_static_group_attention_agrees_with_the_routed_oracle():
+    """Two independently written oracle paths meet: the numpy group attention of Sec. 3.2 fed with
+    the routed groups of a random assignment (queries = keys = the group's tokens) must reproduce
+    the C oracle's per-group attention with unit gates."""
+    rng = np.random.default_rng(8)
+    B, H, N, D, M = 1, 2, 150, 16, 5
+    Q, K, V = (rng.standard_normal((B, H, N, D)).astype(np.float32) for _ in range(3))
+    gid = rng.integers(0, M, (B, N, 1)).astype(np.int32)
+    offsets, perm, _ = oracle.sort(gid, M)
+    groups = [perm[0, offsets[0, g]:offsets[0, g + 1]].astype(np.int64) for g in range(M)]
+    groups = [g for g in groups if len(g)]
+    a = oracle.static_group_attn(Q, K, V, groups, groups, 0.3)
+    b = oracle.attn_all(Q, K, V, gid, np.ones((B, N, 1)), offsets, perm, 0.3)
+    assert np.abs(a - b).max() < 1e-12
