@@ -136,10 +136,6 @@ struct Cfg {
   static constexpr int kDynSmem = kSmemTotal + 1024;      // slack for 1024-byte alignment
 };
 
-struct Shared {   // indices into the mbarrier array
-  int q_full, q_empty, k_full, k_empty, v_full, v_empty, s_full, p_full, o_full, o_empty;
-};
-
 // Output placement.  perm == nullptr: rows stay in sorted order, Op is [B*H, T, D].
 // Otherwise (top-1 routing) the epilogue is the gated inverse permutation of Eq. 5: sorted
 // row p of batch item b goes to token perm[b, p] of O (element strides sb, sh, sn),
