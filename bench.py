@@ -468,7 +468,20 @@ def run_visual_block(mb, cfg, dev, args):
         if it >= args.warmup:
             for i, n in enumerate(names):
                 times[n].append(e[i].elapsed_time(e[i + 1]))
-    for w in (ws, ws_st, ws_fr):
+    # the same block through the single C-ABI call
+    del A, C, Qs, Ks, Vs, Bs
+    st_lists, keep = mb.make_static_lists(lists, F, per_frame, dev)
+    ws_v = mb.alloc_workspace(mb.moga_visual_workspace_bytes(sh, st_lists), dev)
+    one = []
+    for it in range(args.warmup + args.steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        mb.moga_visual_forward(sh, inp["X"], inp["Wr"], inp["bias"], inp["Q"], inp["K"], inp["V"], O, st_lists, ws_v)
+        e1.record()
+        torch.cuda.synchronize()
+        if it >= args.warmup:
+            one.append(e0.elapsed_time(e1))
+    for w in (ws, ws_st, ws_fr, ws_v):
         code, detail = mb.moga_last_device_status(w)
         if code != 0:
             raise RuntimeError(f"device status {code} detail {detail:#x}")
@@ -483,7 +496,7 @@ def run_visual_block(mb, cfg, dev, args):
         "stage": "visual", "config": config_dict(cfg),
         "static_groups": {"frames": F, "windows": [wh, ww], "run_frames": tg, "shot_frames": shot_len, "groups": G,
                           "queries_per_group": [int(nq.min()), int(nq.max())], "keys_per_group": [int(nk.min()), int(nk.max())]},
-        "ms": ms, "ms_total": sum(ms.values()),
+        "ms": ms, "ms_total": sum(ms.values()), "ms_single_call": float(np.mean(one)),
         "st_attn_TFLOP/s": fl_st / ms["st_attn"] / 1e9, "frame_attn_TFLOP/s": fl_fr / ms["frame_attn"] / 1e9,
         "st_gather_GB/s": 2.0 * row * (N + 2 * Tkv) / ms["st_gather"] / 1e6,
         "mean3_GB/s": 4.0 * row * N / ms["mean3"] / 1e6, "hbm_peak_GB/s": peaks["hbm_gbs"],

@@ -230,6 +230,27 @@ moga_status moga_mean3(const moga_shape* s, const void* A, const void* Bs, const
                        const void* C, void* O, void* stream);
 
 /*
+ * The whole visual-attention block of Sec. 3.2 in one call: the routed forward (moga_forward),
+ * the spatial-temporal static branch (gathers by the lists + moga_static_group_attn), the
+ * per-frame branch (one group per latent frame of tokens_per_frame consecutive tokens) and
+ * their mean into O.  `lists` carries DEVICE copies of what moga_stga_build produced, plus
+ * the frame count (F * tokens_per_frame must equal N).  Q, K, V, O contiguous [B, H, N, D]
+ * (non-zero strides: MOGA_ERR_UNSUPPORTED).  ws: at least moga_visual_workspace_bytes; it
+ * holds the forward's workspace, the three branch outputs and the gathered Q / K / V of the
+ * spatial-temporal branch.  The device status word of the routed branch is at the start of
+ * ws (moga_last_device_status(ws, ...)).
+ */
+typedef struct {
+  int32_t G, Tkv;                 /* groups and key rows of the spatial-temporal branch        */
+  int32_t F, tokens_per_frame;    /* latent frames and tokens per frame (per-frame branch)     */
+  const int32_t *q_idx, *q_inv, *q_offsets, *kv_idx, *kv_offsets;   /* device arrays           */
+} moga_static_lists;
+size_t moga_visual_workspace_bytes(const moga_shape* s, const moga_static_lists* lists);
+moga_status moga_visual_forward(const moga_shape* s, const void* X, const float* Wr, const float* bias,
+                                const void* Q, const void* K, const void* V, void* O,
+                                const moga_static_lists* lists, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * "repermute" of Alg. 1 line 4 with the gate of Eq. 5:
  * O[b,h,n,:] = sum_j gate[b,n,j] * Op[b,h,inv[b,n,j],:], summed in fp32 in slot
  * order and rounded once.  No workspace.

@@ -20,7 +20,8 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libmoga.so")
 EXPORTS = ("moga_workspace_bytes", "moga_scratch_bytes", "moga_status_string", "moga_route",
            "moga_permute", "moga_group_attn", "moga_unpermute", "moga_forward",
            "moga_last_device_status", "moga_sort_static", "moga_balance_stats", "moga_stga_build", "moga_gather_rows",
-           "moga_static_group_attn", "moga_mean3", "moga_forward_host_bytes", "moga_forward_host")
+           "moga_static_group_attn", "moga_mean3", "moga_forward_host_bytes", "moga_forward_host",
+           "moga_visual_workspace_bytes", "moga_visual_forward")
 
 MOGA_F32, MOGA_BF16 = 0, 1
 MOGA_ROUTE_AUTO, MOGA_ROUTE_ALU = 0, 1
@@ -38,6 +39,12 @@ class MogaShape(ctypes.Structure):
                 ("route_mode", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
+class MogaStaticLists(ctypes.Structure):
+    _fields_ = [("G", ctypes.c_int32), ("Tkv", ctypes.c_int32), ("F", ctypes.c_int32),
+                ("tokens_per_frame", ctypes.c_int32), ("q_idx", ctypes.c_void_p), ("q_inv", ctypes.c_void_p),
+                ("q_offsets", ctypes.c_void_p), ("kv_idx", ctypes.c_void_p), ("kv_offsets", ctypes.c_void_p)]
+
+
 class MogaError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
@@ -50,7 +57,8 @@ if not os.path.exists(LIB_PATH):
 lib = ctypes.CDLL(LIB_PATH)
 for _n in EXPORTS:
     getattr(lib, _n).restype = ctypes.c_int
-for _n in ("moga_workspace_bytes", "moga_scratch_bytes", "moga_static_scratch_bytes", "moga_forward_host_bytes"):
+for _n in ("moga_workspace_bytes", "moga_scratch_bytes", "moga_static_scratch_bytes", "moga_forward_host_bytes",
+           "moga_visual_workspace_bytes"):
     getattr(lib, _n).restype = ctypes.c_size_t
 lib.moga_status_string.restype = ctypes.c_char_p
 
@@ -187,6 +195,25 @@ def moga_forward_host(shape, X, Wr, bias, Q, K, V, O, arena, heads_per_chunk, gi
                                  _ptr(O), _ptr(gid_out), _ptr(gate_out), _ptr(arena),
                                  ctypes.c_size_t(arena.numel()), ctypes.c_int32(heads_per_chunk), _stream()),
            "moga_forward_host")
+
+
+def make_static_lists(lists, F, tokens_per_frame, device="cuda"):
+    """Device copies of moga_stga_build's arrays wrapped for moga_visual_forward.  Returns the
+    ctypes struct and the tensors that keep the device memory alive."""
+    keep = {k: torch.from_numpy(lists[k]).to(device) for k in ("q_idx", "q_inv", "q_offsets", "kv_idx", "kv_offsets")}
+    st = MogaStaticLists(lists["G"], lists["Tkv"], F, tokens_per_frame, *(keep[k].data_ptr() for k in
+                         ("q_idx", "q_inv", "q_offsets", "kv_idx", "kv_offsets")))
+    return st, keep
+
+
+def moga_visual_workspace_bytes(shape, static_lists) -> int:
+    return int(lib.moga_visual_workspace_bytes(ctypes.byref(shape), ctypes.byref(static_lists)))
+
+
+def moga_visual_forward(shape, X, Wr, bias, Q, K, V, O, static_lists, ws):
+    _check(lib.moga_visual_forward(ctypes.byref(shape), _ptr(X), _ptr(Wr), _ptr(bias), _ptr(Q), _ptr(K), _ptr(V),
+                                   _ptr(O), ctypes.byref(static_lists), _ptr(ws), ctypes.c_size_t(ws.numel()),
+                                   _stream()), "moga_visual_forward")
 
 
 def moga_last_device_status(ws):

@@ -279,6 +279,78 @@ moga_status moga_forward(const moga_shape* s, const void* X, const float* Wr, co
   return MOGA_OK;
 }
 
+// ---- the whole visual-attention block (Sec. 3.2): routed branch + two static branches + mean
+namespace {
+struct VisualLayout {
+  size_t fwd, st_scratch, fr_scratch, fr_off, A, C, Qs, Ks, Vs, Bs, total;
+};
+VisualLayout visual_layout(const moga_shape& s, int G, int Tkv, int F) {
+  VisualLayout v{};
+  const size_t es = elem_size(s.dtype), row = es * (size_t)s.B * s.H * s.D;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = off;
+    off = align_up(off + bytes, kWsAlign);
+    return at;
+  };
+  v.fwd = take(ws_layout(s).total);
+  v.st_scratch = take(moga_static_scratch_bytes(&s, G));
+  v.fr_scratch = take(moga_static_scratch_bytes(&s, F));
+  v.fr_off = take(sizeof(int32_t) * ((size_t)F + 1));
+  v.A = take(row * s.N);
+  v.C = take(row * s.N);
+  v.Qs = take(row * s.N);
+  v.Ks = take(row * Tkv);
+  v.Vs = take(row * Tkv);
+  v.Bs = take(row * s.N);
+  v.total = off;
+  return v;
+}
+bool lists_ok(const moga_shape& s, const moga_static_lists* l) {
+  return l != nullptr && l->G >= 1 && l->Tkv >= 1 && l->F >= 1 && l->tokens_per_frame >= 1 &&
+         (long long)l->F * l->tokens_per_frame == s.N && l->q_idx && l->q_inv && l->q_offsets && l->kv_idx &&
+         l->kv_offsets;
+}
+}  // namespace
+
+size_t moga_visual_workspace_bytes(const moga_shape* s, const moga_static_lists* lists) {
+  moga_status st;
+  if (!check_shape(s, &st) || !lists_ok(*s, lists)) return 0;
+  return visual_layout(*s, lists->G, lists->Tkv, lists->F).total;
+}
+
+moga_status moga_visual_forward(const moga_shape* s, const void* X, const float* Wr, const float* bias,
+                                const void* Q, const void* K, const void* V, void* O,
+                                const moga_static_lists* lists, void* ws, size_t ws_bytes, void* stream) {
+  moga_status st;
+  if (!check_shape(s, &st)) return st;
+  if (!lists_ok(*s, lists)) return MOGA_ERR_INVALID_ARG;
+  if (s->q_stride_b || s->q_stride_h || s->q_stride_n) return MOGA_ERR_UNSUPPORTED;   // per-frame branch reads Q, K, V in place
+  const VisualLayout v = visual_layout(*s, lists->G, lists->Tkv, lists->F);
+  if (!check_ws(ws, ws_bytes, v.total, &st)) return st;
+  char* w = static_cast<char*>(ws);
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  // routed branch -> A
+  st = moga_forward(s, X, Wr, bias, Q, K, V, w + v.A, nullptr, nullptr, nullptr, nullptr, w + v.fwd,
+                    ws_layout(*s).total, stream);
+  if (st != MOGA_OK) return st;
+  // spatial-temporal branch -> Bs (query order of the lists)
+  if ((st = launch_gather_list(*s, lists->q_idx, s->N, Q, w + v.Qs, cs)) != MOGA_OK) return st;
+  if ((st = launch_gather_list(*s, lists->kv_idx, lists->Tkv, K, w + v.Ks, cs)) != MOGA_OK) return st;
+  if ((st = launch_gather_list(*s, lists->kv_idx, lists->Tkv, V, w + v.Vs, cs)) != MOGA_OK) return st;
+  st = moga_static_group_attn(s, lists->G, s->N, lists->Tkv, w + v.Qs, w + v.Ks, w + v.Vs, lists->q_offsets,
+                              lists->kv_offsets, w + v.Bs, nullptr, w + v.st_scratch,
+                              moga_static_scratch_bytes(s, lists->G), stream);
+  if (st != MOGA_OK) return st;
+  // per-frame branch -> C (token order: a frame's tokens are contiguous)
+  int32_t* fr_off = reinterpret_cast<int32_t*>(w + v.fr_off);
+  if ((st = launch_frame_offsets(fr_off, lists->F, lists->tokens_per_frame, cs)) != MOGA_OK) return st;
+  st = moga_static_group_attn(s, lists->F, s->N, s->N, Q, K, V, fr_off, fr_off, w + v.C, nullptr, w + v.fr_scratch,
+                              moga_static_scratch_bytes(s, lists->F), stream);
+  if (st != MOGA_OK) return st;
+  return launch_mean3(*s, w + v.A, w + v.Bs, lists->q_inv, w + v.C, O, cs);
+}
+
 moga_status moga_last_device_status(void* ws, void* stream, uint32_t* detail) {
   if (ws == nullptr) return MOGA_ERR_WORKSPACE;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);

@@ -112,6 +112,7 @@ moga_status launch_attn_f32_groups(int B, int H, int D, float scale, int G, int 
                                    cudaStream_t st);
 moga_status launch_gather_list(const moga_shape& s, const int32_t* idx, int L, const void* src, void* dst,
                                cudaStream_t st);
+moga_status launch_frame_offsets(int32_t* off, int F, int tokens_per_frame, cudaStream_t st);
 moga_status launch_mean3(const moga_shape& s, const void* A, const void* Bs, const int32_t* inv_b, const void* C,
                          void* O, cudaStream_t st);
 moga_status stga_build_host(int F, int Hh, int Ww, int wh, int ww, const int32_t* shot_starts, int n_shots,

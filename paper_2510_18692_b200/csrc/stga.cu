@@ -90,7 +90,18 @@ mean3_kernel(const uint4* __restrict__ A, const uint4* __restrict__ Bs, const in
   }
 }
 
+// off[f] = f * tokens_per_frame, f = 0..F: the per-frame groups (queries = keys)
+__global__ void frame_offsets_kernel(int32_t* __restrict__ off, int F, int tokens_per_frame) {
+  for (int f = blockIdx.x * blockDim.x + threadIdx.x; f <= F; f += gridDim.x * blockDim.x) off[f] = f * tokens_per_frame;
+}
+
 }  // namespace
+
+moga_status launch_frame_offsets(int32_t* off, int F, int tokens_per_frame, cudaStream_t st) {
+  frame_offsets_kernel<<<(F + 256) / 256, 256, 0, st>>>(off, F, tokens_per_frame);
+  MOGA_CUDA_OK(cudaGetLastError());
+  return MOGA_OK;
+}
 
 moga_status launch_gather_list(const moga_shape& s, const int32_t* idx, int L, const void* src, void* dst,
                                cudaStream_t st) {

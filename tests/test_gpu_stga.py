@@ -139,6 +139,13 @@ def test_visual_attention_block(mb, dtype):
     oC = oracle.static_group_attn(host["Q"], host["K"], host["V"], fq, fk, cfg.scale)
     check_output(C.float().cpu().numpy(), oC, dtype, "frame branch")
     check_output(O.float().cpu().numpy(), oracle.mean3(oA, oB, oC), dtype, "mean of three")
+    # the same block through the single entry point: the same kernels, so the same bits
+    st_lists, keep = mb.make_static_lists(lists, F, Hh * Ww)
+    ws_v = mb.alloc_workspace(mb.moga_visual_workspace_bytes(sh, st_lists))
+    O1 = torch.full_like(O, float("nan"))
+    mb.moga_visual_forward(sh, inp["X"], inp["Wr"], None, inp["Q"], inp["K"], inp["V"], O1, st_lists, ws_v)
+    assert mb.moga_last_device_status(ws_v) == (0, 0)
+    assert torch.equal(O1, O)
     # the combine step alone, against the mean of the GPU's own branch outputs (fp32 sum, one rounding)
     Bt = Bs[:, :, torch.from_numpy(lists["q_inv"].astype(np.int64)).cuda()]
     ref = (A.double() + Bt.double() + C.double()) / 3
