@@ -370,7 +370,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       const int tile_row0 = it.row0 + x * kTileM;
       float m = -INFINITY, l = 0.f;
       for (int j = 0; j < ntiles && ok; ++j) {
-        ok = wait(S_FULL + x, n_s & 1u, 10);
+        ok = __all_sync(0xffffffffu, wait(S_FULL + x, n_s & 1u, 10));   // warp-uniform: TMEM loads are warp-collective
         if (!ok) break;
         ++n_s;
         tc_fence_after();
@@ -444,7 +444,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       }
       if (!ok) break;
       // ---- epilogue: O / l -> bf16 -> per-warp staging -> global
-      ok = wait(O_FULL + x, n_o & 1u, 11);
+      ok = __all_sync(0xffffffffu, wait(O_FULL + x, n_o & 1u, 11));
       if (!ok) break;
       ++n_o;
       tc_fence_after();

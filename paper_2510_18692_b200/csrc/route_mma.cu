@@ -183,7 +183,7 @@ route_mma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
     uint32_t nt = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < ntiles; tile += gridDim.x, ++nt) {
-      ok = wait(ACC_FULL, nt & 1u, 4);
+      ok = __all_sync(0xffffffffu, wait(ACC_FULL, nt & 1u, 4));   // warp-uniform: TMEM loads are warp-collective
       if (!ok) break;
       tc_fence_after();
       float r[MP];
