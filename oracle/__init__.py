@@ -224,6 +224,25 @@ def static_group_attn(Q, K, V, q_groups, kv_groups, scale):
     return O
 
 
+def static_group_attn_rows(Q, K, V, q_groups, kv_groups, scale, rows):
+    """Eq. 1 inside caller-given groups for the listed (b, h, token) rows only, one row at a
+    time from the definition: scores of the token's query against the keys of the group that
+    owns it, max-subtracted softmax, weighted sum of that group's values.  fp64 [nrows, D].
+    Serves the paper-sized static-branch comparisons, where the full tensor of
+    static_group_attn is out of reach on the host."""
+    owner = {}
+    for g, qi in enumerate(q_groups):
+        for n in qi:
+            owner[int(n)] = g
+    out = np.empty((len(rows), Q.shape[-1]))
+    for i, (b, h, n) in enumerate(rows):
+        ki = kv_groups[owner[int(n)]]
+        s = (np.asarray(K[b, h, ki], dtype=np.float64) @ np.asarray(Q[b, h, n], dtype=np.float64)) * scale
+        p = np.exp(s - s.max())
+        out[i] = (p / p.sum()) @ np.asarray(V[b, h, ki], dtype=np.float64)
+    return out
+
+
 def mean3(a, b, c):
     """Sec. 3.2: a token's output is the mean of its dynamic (MoGA) and two static group outputs."""
     return (np.asarray(a, np.float64) + np.asarray(b, np.float64) + np.asarray(c, np.float64)) / 3.0

@@ -54,14 +54,41 @@ def check_sort(gid_gpu, perm, inv, offsets, M):
     return o_off, o_perm, o_inv
 
 
+# Relative bounds, beside the absolute ones above.  With N(0, 1) inputs and groups of ~17,000 keys
+# the outputs are of the order 1e-3, below the absolute bounds, so those alone would accept an
+# output that is scaled or zero.  REL_FRO bounds ||got - want||_F / ||want||_F over the whole
+# comparison; ROW bounds each row's largest error by a fraction of that row's largest magnitude
+# (bf16: 2^-6, i.e. a few units in the last place of the 8-bit mantissa after two roundings).
+REL_FRO = {"bf16": 1e-2, "f32": 1e-5}
+ROW_REL = {"bf16": 2.0 ** -6, "f32": 2.0 ** -16}
+ROW_ABS = 1e-5
+
+
 def check_output(got, want, dtype, what="O"):
+    """Absolute bounds (max, mean), the relative Frobenius error and a per-row relative bound;
+    rows are the last axis.  Returns (max abs err, mean abs err, relative Frobenius err)."""
     got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    assert got.shape == want.shape, f"{what}: shape {got.shape} vs {want.shape}"
+    if got.size == 0:
+        return 0.0, 0.0, 0.0
     err = np.abs(got - want)
     tol = TOL[dtype]
     assert np.all(np.isfinite(got)), f"{what}: non-finite values"
     assert err.max(initial=0.0) <= tol["max_abs"], f"{what}: max abs err {err.max():.3e}"
     assert err.mean() <= tol["mean_abs"], f"{what}: mean abs err {err.mean():.3e}"
-    return float(err.max(initial=0.0)), float(err.mean())
+    norm = float(np.sqrt((want ** 2).sum()))
+    rel = float(np.sqrt((err ** 2).sum())) / norm if norm > 0 else float(err.max() > 0)
+    assert rel <= REL_FRO[dtype], f"{what}: relative Frobenius err {rel:.3e}"
+    row_err = err.reshape(-1, err.shape[-1]).max(axis=1)
+    row_mag = np.abs(want).reshape(-1, want.shape[-1]).max(axis=1)
+    excess = row_err - (ROW_REL[dtype] * row_mag + ROW_ABS)
+    worst = int(np.argmax(excess))
+    assert excess[worst] <= 0, (f"{what}: row {worst}: err {row_err[worst]:.3e} against row magnitude "
+                                f"{row_mag[worst]:.3e}")
+    print(f"{what}: max abs {err.max():.3e}  mean abs {err.mean():.3e}  rel fro {rel:.3e}  "
+          f"worst row err/mag {float((row_err / np.maximum(row_mag, 1e-30)).max()):.3e}")
+    return float(err.max(initial=0.0)), float(err.mean()), rel
 
 
 def grouped_case(sizes, H, D, dtype, seed, B=1, qscale=1.0, device="cuda"):

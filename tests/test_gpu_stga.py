@@ -153,21 +153,6 @@ def test_visual_attention_block(mb, dtype):
     assert (O.double() - ref).abs().max().item() <= tol
 
 
-def _static_rows_oracle(Q, K, V, q_groups, kv_groups, scale, rows):
-    """fp64 rows of the static group attention, one (b, h, token) at a time, from the definition."""
-    owner = {}
-    for g, qi in enumerate(q_groups):
-        for n in qi:
-            owner[int(n)] = g
-    out = np.empty((len(rows), Q.shape[-1]))
-    for i, (b, h, n) in enumerate(rows):
-        ki = kv_groups[owner[int(n)]]
-        s = (K[b, h, ki].astype(np.float64) @ Q[b, h, n].astype(np.float64)) * scale
-        p = np.exp(s - s.max())
-        out[i] = (p / p.sum()) @ V[b, h, ki].astype(np.float64)
-    return out
-
-
 @pytest.mark.parametrize("name", ["clip_bf16", "minute_bf16"])
 def test_static_branches_full_size_sampled(mb, name):
     """The static branches in the configuration bench.py --stage visual times (4 x 4 windows, runs of
@@ -203,9 +188,9 @@ def test_static_branches_full_size_sampled(mb, name):
     rows = [(0, h, n) for n in toks for h in heads]
     Qh, Kh, Vh = (to_np32(inp[n][:, heads]) for n in ("Q", "K", "V"))
     rows_h = [(b, heads.index(h), n) for b, h, n in rows]
-    want_st = _static_rows_oracle(Qh, Kh, Vh, qg, kg, cfg.scale, rows_h)
+    want_st = oracle.static_group_attn_rows(Qh, Kh, Vh, qg, kg, cfg.scale, rows_h)
     fq, fk = oracle.frame_groups(F, Hh, Ww)
-    want_fr = _static_rows_oracle(Qh, Kh, Vh, fq, fk, cfg.scale, rows_h)
+    want_fr = oracle.static_group_attn_rows(Qh, Kh, Vh, fq, fk, cfg.scale, rows_h)
     q_inv = torch.from_numpy(lists["q_inv"].astype(np.int64)).cuda()
     bi = torch.tensor([r[0] for r in rows]).cuda()
     hi = torch.tensor([r[1] for r in rows]).cuda()
