@@ -34,10 +34,24 @@ if ROOT not in sys.path:
 from paper_2510_18692_b200.inputs import CONFIGS, make_inputs, useful_flops  # noqa: E402
 
 METRIC = "MoGA fwd effective TFLOP/s (bf16)"
+L2_FLUSH_BYTES = 256 << 20           # twice the 126 MB L2
+SM_COUNT, FP32_LANES_PER_SM = 148, 128   # B200: fp32 FMA peak = SMs x lanes x 2 flop x clock
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes of the attention kernel / its algorithmic bytes, from the ncu capture of the current
-# kernel summarised in profiles/attn_bf16_kernel_clip_bf16_ncu_full.md (traffic grows with T*H).
-ATTN_TRAFFIC_RATIO = 0.958
+# DRAM bytes of the attention kernel / its algorithmic bytes, from the ncu capture of the
+# clip-sized case (traffic grows with T*H: every Q/K/V/O byte crosses DRAM once).  The figure
+# belongs to one version of the kernel source: when the source's hash differs, traffic is null.
+ATTN_TRAFFIC = {"ratio": 0.958, "source_sha16": "@@SHA@@"}
+
+
+def attn_traffic_ratio():
+    import hashlib
+    path = os.path.join(ROOT, "paper_2510_18692_b200", "csrc", "attn_bf16.cu")
+    try:
+        with open(path, "rb") as f:
+            sha = hashlib.sha256(f.read()).hexdigest()[:16]
+    except OSError:
+        return None
+    return ATTN_TRAFFIC["ratio"] if sha == ATTN_TRAFFIC["source_sha16"] else None
 
 
 def kernels_per_forward(cfg):
@@ -91,15 +105,21 @@ class ClockSampler:
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
-        self.index = index
+    def __init__(self, device):
+        """`device`: a torch CUDA device.  The GPU is named to nvidia-smi by its UUID: the CUDA
+        ordinal is not the physical index once CUDA_VISIBLE_DEVICES is set."""
+        try:
+            self.uuid = "GPU-" + str(torch.cuda.get_device_properties(device).uuid).removeprefix("GPU-")
+        except Exception:   # noqa: BLE001  (older torch without the field)
+            self.uuid = None
+        self.index = str(device.index or 0) if self.uuid is None else self.uuid
         self.proc = None
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
-                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-i", self.index], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
 
@@ -127,7 +147,7 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons), "gpu_uuid": self.uuid}
 
 
 # ----------------------------------------------------------------------------- CPU oracle legs
@@ -195,16 +215,19 @@ def run_reference(args, cfg):
 
 
 def config_dict(cfg):
+    es = 2 if cfg.dtype == "bf16" else 4
+    resident = cfg.B * cfg.N * (cfg.C + 3 * cfg.H * cfg.D) * es
     return {"workload": cfg.name, "B": cfg.B, "H": cfg.H, "N": cfg.N, "C": cfg.C, "D": cfg.D, "M": cfg.M,
             "k": cfg.k, "gate_mode": "softmax_all" if cfg.gate_mode == 0 else "softmax_topk",
-            "l2": "inputs larger than L2 (no flush needed)"}
+            "l2": "inputs larger than L2 (no flush needed)" if resident >= L2_FLUSH_BYTES
+                  else "L2 flushed before every timed step (a 256 MB buffer rewritten)"}
 
 
 # ----------------------------------------------------------------------------- GPU arm
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="minute_bf16", choices=sorted(CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -265,16 +288,26 @@ def main():
     sizes = np.diff(offsets.cpu().numpy(), axis=1)
     flops = sum(useful_flops(sizes[b], cfg.H, cfg.D) for b in range(cfg.B))
 
-    clocks = ClockSampler(local_rank)
+    clocks = ClockSampler(dev)
     clocks.start()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    # exactly args.steps steps between two synchronisations, each between its own pair of events
+    # (the headline is the median of the per-step times; their mean is kept beside it).  Inputs
+    # smaller than L2 would stay cached from step to step: then a buffer larger than L2 is
+    # rewritten before every step, outside that step's event pair.
+    resident = sum(inp[n].numel() * inp[n].element_size() for n in ("X", "Q", "K", "V"))
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev) if resident < L2_FLUSH_BYTES else None
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     barrier_sync()
-    ev[0].record()
-    for _ in range(args.steps):
+    for e0, e1 in ev:
+        if flush is not None:
+            flush.fill_(1)
+        e0.record()
         step()
-    ev[1].record()
+        e1.record()
     barrier_sync()
-    ms_local = ev[0].elapsed_time(ev[1]) / args.steps
+    per_step = [e0.elapsed_time(e1) for e0, e1 in ev]
+    ms_mean_local = float(np.mean(per_step))
+    ms_local = float(statistics.median(per_step))
 
     # per-stage breakdown through the stage entry points (same kernels, same data)
     es = 2 if cfg.dtype == "bf16" else 4
@@ -283,6 +316,8 @@ def main():
     stage_ms = {n: [] for n in stage_names}
     for it in range(args.steps + 1):
         e = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+        if flush is not None:
+            flush.fill_(1)
         e[0].record()
         mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], gid, gate, None, ws)
         e[1].record()
@@ -298,9 +333,10 @@ def main():
                 stage_ms[n].append(e[i].elapsed_time(e[i + 1]))
     clk = clocks.stop()
     del Qp, Kp, Vp, Op
-    stage = {n: float(np.mean(v)) for n, v in stage_ms.items()}
+    stage = {n: float(statistics.median(v)) for n, v in stage_ms.items()}
 
     ms, total_flops = aggregate(ms_local, flops, dev)
+    ms_mean, _ = aggregate(ms_mean_local, flops, dev)
     value = total_flops / (ms * 1e-3) / 1e12
     peaks = load_peaks()
     attn_tflops = flops / (stage["group_attn"] * 1e-3) / 1e12
@@ -314,23 +350,42 @@ def main():
     for n, by in bytes_alg.items():
         gbs = by / (stage[n] * 1e-3) / 1e9
         stages_out[n].update({"GB/s": gbs, "frac_hbm": gbs / peaks["hbm_gbs"]})
+    mhz = clk.get("sm_mhz")
     stages_out["group_attn"].update({"TFLOP/s": attn_tflops,
-                                     "frac_tensor_burst": attn_tflops / peaks["bf16_tflops"]})
+                                     "frac_tensor_burst": attn_tflops / peaks["bf16_tflops"],
+                                     "frac_tensor_sustained": attn_tflops / peaks["bf16_tflops_sustained"],
+                                     # time x clock: compares boxes whose power cap settles at different clocks
+                                     "ms_x_sm_mhz": None if not mhz else stage["group_attn"] * mhz})
+    ratio = attn_traffic_ratio() if cfg.dtype == "bf16" else None
     out = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": ms, "ms_per_step_mean": ms_mean,
+        "timing": f"median of {args.steps} per-step CUDA-event times (max over ranks); mean over the region beside it",
+        "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic", "config": config_dict(cfg),
+        "route_kernel": "tensor" if cfg.dtype == "bf16" else "alu",
         "ms_per_layer_head_batch": ms / (cfg.B * cfg.H), "useful_tflop_per_step": flops / 1e12,
         "group_sizes": {"min": int(sizes.min()), "max": int(sizes.max()), "empty": int((sizes == 0).sum())},
         "stages": stages_out, "gpu_launches": kernels_per_forward(cfg) * args.steps, "clocks": clk,
-        "roofline": {"kernel": "moga_group_attn (tcgen05 varlen attention)", "bound": "tensor",
-                     "achieved": attn_tflops, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                     "frac": attn_tflops / peaks["bf16_tflops_sustained"],
-                     "peak_source": f"{peaks['source']} sustained bf16 GEMM",
-                     "frac_of_burst_peak": attn_tflops / peaks["bf16_tflops"],
-                     "traffic": ATTN_TRAFFIC_RATIO * 4.0 * tok * cfg.k * cfg.H * cfg.D * es if cfg.dtype == "bf16" else None,
-                     "traffic_unit": "bytes per launch (ncu dram bytes of the clip_bf16 capture, scaled by T*H)"},
     }
+    if cfg.dtype == "bf16":
+        out["roofline"] = {
+            "kernel": "moga_group_attn (tcgen05 varlen attention)", "bound": "tensor",
+            "achieved": attn_tflops, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+            "frac": attn_tflops / peaks["bf16_tflops_sustained"],
+            "peak_source": f"{peaks['source']} sustained bf16 GEMM",
+            "frac_of_burst_peak": attn_tflops / peaks["bf16_tflops"],
+            "algorithmic_bytes": 4.0 * tok * cfg.k * cfg.H * cfg.D * es,
+            "traffic": None if ratio is None else ratio * 4.0 * tok * cfg.k * cfg.H * cfg.D * es,
+            "traffic_unit": "bytes per launch (ncu dram bytes of the clip_bf16 capture, scaled by T*H; "
+                            "null when the kernel source changed after the capture)"}
+    else:
+        # fp32 attention runs on the fp32 ALUs: 2 flop per lane per clock at the maximum SM clock
+        alu_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * (clk.get("sm_max_mhz") or peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
+        out["roofline"] = {
+            "kernel": "moga_group_attn (fp32 ALU varlen attention)", "bound": "alu", "achieved": attn_tflops,
+            "peak": alu_peak, "unit": "TFLOP/s", "frac": attn_tflops / alu_peak,
+            "peak_source": "148 SMs x 128 fp32 lanes x 2 flop x max SM clock", "traffic": None}
 
     if rank == 0 and not args.no_e2e:
         out["e2e"] = run_e2e(mb, cfg, sh, inp, ws, O, flops, args)
@@ -396,7 +451,7 @@ def run_head_sharded(mb, cfg, dev, args, rank, world):
         _, _, offsets = step()
     sizes = np.diff(offsets.cpu().numpy(), axis=1)
     flops_local = sum(useful_flops(sizes[b], h_hi - h_lo, cfg.D) for b in range(cfg.B))
-    clocks = ClockSampler(dev.index or 0)
+    clocks = ClockSampler(dev)
     clocks.start()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
     barrier_sync()

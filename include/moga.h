@@ -152,6 +152,8 @@ moga_status moga_permute(const moga_shape* s, const int32_t* gid, const void* Q,
  *  - status_out, if non-NULL, is a device pointer to two uint32 (8-byte aligned) that
  *    receives {status, detail} as moga_last_device_status would report them, e.g.
  *    MOGA_ERR_INTERNAL for a gid outside [0, M) (which is clamped).
+ *  - N = 0 is valid as everywhere else: offsets are set to zero, gid / perm / inv may be
+ *    NULL, the array is not touched.
  */
 moga_status moga_sort_static(const moga_shape* s, const int32_t* gid, int32_t* perm, int32_t* inv,
                              int32_t* offsets, uint32_t* status_out, void* stream);
@@ -299,6 +301,21 @@ moga_status moga_forward_host(const moga_shape* s, const void* X, const float* W
  * `detail`, if non-NULL, receives a kernel-specific word saying where.
  */
 moga_status moga_last_device_status(void* ws, void* stream, uint32_t* detail);
+
+/*
+ * Self-test of the time-out path (the paper has no counterpart: it is a diagnostic).
+ * Every wait inside the tensor-core kernels is bounded; when one runs out the kernel writes
+ * MOGA_ERR_TIMEOUT and a detail word to the status header and returns normally.  This call
+ * runs that same wait routine to its limit in a one-block kernel of its own, on a barrier
+ * nothing signals, so a deployment can check that a stuck wait is reported rather than hung.
+ * ws: device memory, >= 256 bytes, 256-byte aligned (any workspace of this library will do;
+ * its status header is reset).  limit_ns: the bound of the wait, 1 .. 100,000,000 (100 ms),
+ * else MOGA_ERR_INVALID_ARG.  Asynchronous on `stream`.  Afterwards moga_last_device_status(ws)
+ * returns MOGA_ERR_TIMEOUT with detail = 0x7e000000 | (block << 8) | barrier index (both 0
+ * here); words 2-3 of the header hold the nanoseconds the wait lasted and word 4 how the
+ * second warp left (1: released by the abort flag).
+ */
+moga_status moga_selftest_wait_timeout(void* ws, size_t ws_bytes, uint64_t limit_ns, void* stream);
 
 #ifdef __cplusplus
 }

@@ -21,7 +21,7 @@ EXPORTS = ("moga_workspace_bytes", "moga_scratch_bytes", "moga_status_string", "
            "moga_permute", "moga_group_attn", "moga_unpermute", "moga_forward",
            "moga_last_device_status", "moga_sort_static", "moga_balance_stats", "moga_stga_build", "moga_gather_rows",
            "moga_static_group_attn", "moga_mean3", "moga_forward_host_bytes", "moga_forward_host",
-           "moga_visual_workspace_bytes", "moga_visual_forward")
+           "moga_visual_workspace_bytes", "moga_visual_forward", "moga_selftest_wait_timeout")
 
 MOGA_F32, MOGA_BF16 = 0, 1
 MOGA_ROUTE_AUTO, MOGA_ROUTE_ALU = 0, 1
@@ -214,6 +214,11 @@ def moga_visual_forward(shape, X, Wr, bias, Q, K, V, O, static_lists, ws):
     _check(lib.moga_visual_forward(ctypes.byref(shape), _ptr(X), _ptr(Wr), _ptr(bias), _ptr(Q), _ptr(K), _ptr(V),
                                    _ptr(O), ctypes.byref(static_lists), _ptr(ws), ctypes.c_size_t(ws.numel()),
                                    _stream()), "moga_visual_forward")
+
+
+def moga_selftest_wait_timeout(ws, limit_ns):
+    _check(lib.moga_selftest_wait_timeout(_ptr(ws), ctypes.c_size_t(ws.numel()), ctypes.c_uint64(limit_ns),
+                                          _stream()), "moga_selftest_wait_timeout")
 
 
 def moga_last_device_status(ws):

@@ -25,6 +25,8 @@
 #include "moga_internal.cuh"
 #include "sm100_ptx.cuh"
 
+#include <type_traits>
+
 namespace moga {
 namespace {
 
@@ -32,7 +34,6 @@ constexpr int kThreads = 384;
 constexpr int kTileM = 128;       // query rows per tile
 constexpr int kTileN = 128;       // keys per K/V tile
 constexpr int kQBlock = 2 * kTileM;
-constexpr uint64_t kWaitLimitNs = 4000000000ull;  // 4 s: far above any legitimate wait
 constexpr float kRowSumLimit = 1.0995116e12f;      // 2^40: a tile's row sum beyond this forces a new maximum
 
 using namespace sm100;
@@ -153,7 +154,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                  const __grid_constant__ CUtensorMap mapV, const Groups grp,
                  const int32_t* __restrict__ order, const int32_t* __restrict__ prefix,
                  __nv_bfloat16* __restrict__ Op, float* __restrict__ lse, uint32_t* header, int T, int H,
-                 int BG, float scale_log2, float scale, const Scatter sc) {
+                 int BG, float scale_log2, float scale, const Scatter sc, uint64_t wait_limit_ns) {
   using C = Cfg<D>;
   constexpr int NS = C::NS;
   extern __shared__ unsigned char smem_raw[];
@@ -205,21 +206,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 
   // Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
   auto wait = [&](int idx, uint32_t parity, uint32_t where) -> bool {
-    const uint32_t b = bar(idx);
-    if (mbar_try_wait(b, parity)) return true;
-    const uint64_t t0 = global_timer_ns();
-    uint32_t spins = 0;
-    while (!mbar_try_wait(b, parity)) {
-      if ((++spins & 255u) == 0) {
-        if (*abort_flag) return false;
-        if (global_timer_ns() - t0 > kWaitLimitNs) {
-          *abort_flag = 1;
-          report_status(header, MOGA_ERR_TIMEOUT, (where << 24) | ((uint32_t)blockIdx.x << 8) | (uint32_t)idx);
-          return false;
-        }
-      }
-    }
-    return true;
+    const WaitResult res = mbar_wait_bounded(bar(idx), parity, abort_flag, wait_limit_ns);
+    if (res == kWaitExpired)
+      report_status(header, MOGA_ERR_TIMEOUT, (where << 24) | ((uint32_t)blockIdx.x << 8) | (uint32_t)idx);
+    return res == kWaitDone;
   };
 
   // Registers move from the producer / MMA warpgroup (warps 0-3) to the softmax warpgroups:
@@ -361,12 +351,14 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     const uint32_t tS = tmem + lane_off + x * kTileN;
     const uint32_t tO = tmem + lane_off + 256 + x * 128;
-    uint32_t n_s = 0, n_o = 0;
+    uint32_t n_s = 0, n_o = 0, n_kv = 0;             // n_kv: K/V tiles of earlier items (ring position)
     bool ok = true;
     for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
       const Item it = decode_item(w, grp, order, prefix, BG, H);
-      if (x == 1 && !(it.row0 + kTileM < it.qhi)) continue;
       const int ntiles = (it.khi - it.klo + kTileN - 1) / kTileN;
+      const uint32_t kv0 = n_kv;
+      n_kv += (uint32_t)ntiles;
+      if (x == 1 && !(it.row0 + kTileM < it.qhi)) continue;
       const int tile_row0 = it.row0 + x * kTileM;
       float m = -INFINITY, l = 0.f;
       for (int j = 0; j < ntiles && ok; ++j) {
@@ -388,7 +380,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 #pragma unroll
           for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
           tmem_wait_ld();
-          if (ncols < kTileN) {
+          const bool ragged = ncols < kTileN;
+          if (ragged && exact) {
+            // columns past the group's last key hold scores against the next group's rows:
+            // keep them out of the maximum (comparisons only, so scale = 0 cannot make a NaN)
 #pragma unroll
             for (int c = 0; c < 128; ++c)
               if (c >= ncols) sreg[c] = 0xff800000u;        // -inf
@@ -409,15 +404,24 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
           const float neg_m = -m * scale_log2;
           const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(neg_m, neg_m);
           float2 ls[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+          // p = 2^(s * scale_log2 - m * scale_log2); on a ragged tile the weight of a column past
+          // the last key is an exact 0 selected after the exponential, whatever its score holds
+          auto weights = [&](auto masked) {
 #pragma unroll
-          for (int c = 0; c < 64; ++c) {
-            const float2 x = __ffma2_rn(make_float2(__uint_as_float(sreg[2 * c]), __uint_as_float(sreg[2 * c + 1])),
-                                        sc2, nm2);
-            const float2 pe = make_float2(ex2(x.x), ex2(x.y));
-            ls[c & 3] = __fadd2_rn(ls[c & 3], pe);
-            __nv_bfloat162 pk = __floats2bfloat162_rn(pe.x, pe.y);
-            preg[c] = *reinterpret_cast<uint32_t*>(&pk);
-          }
+            for (int c = 0; c < 64; ++c) {
+              const float2 x = __ffma2_rn(make_float2(__uint_as_float(sreg[2 * c]), __uint_as_float(sreg[2 * c + 1])),
+                                          sc2, nm2);
+              float2 pe = make_float2(ex2(x.x), ex2(x.y));
+              if (decltype(masked)::value) {
+                pe.x = 2 * c < ncols ? pe.x : 0.f;
+                pe.y = 2 * c + 1 < ncols ? pe.y : 0.f;
+              }
+              ls[c & 3] = __fadd2_rn(ls[c & 3], pe);
+              __nv_bfloat162 pk = __floats2bfloat162_rn(pe.x, pe.y);
+              preg[c] = *reinterpret_cast<uint32_t*>(&pk);
+            }
+          };
+          if (ragged) weights(std::true_type{}); else weights(std::false_type{});
           const float2 l01 = __fadd2_rn(__fadd2_rn(ls[0], ls[1]), __fadd2_rn(ls[2], ls[3]));
           lsum = l01.x + l01.y;
           if (exact || !__any_sync(0xffffffffu, !(lsum < kRowSumLimit))) break;
@@ -426,6 +430,24 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         l = l * alpha + lsum;
         tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&preg[0]));
         tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&preg[32]));
+        if (x == 0 && ncols < kTileN) {
+          // Ragged last tile: the V rows past the group's last key belong to the next group (or
+          // are the zero fill past T).  Their weights are 0, but 0 x inf would still poison O, so
+          // tile A's warps clear those rows in shared memory before either tile's P V is issued
+          // (the MMA warp waits for P_FULL of tile A first).  Thread r owns key row r.
+          const uint32_t slot = (kv0 + (uint32_t)j) % NS;
+          ok = __all_sync(0xffffffffu, wait(V_FULL + slot, ((kv0 + (uint32_t)j) / NS) & 1u, 12));
+          if (!ok) break;
+          if (r >= ncols) {
+#pragma unroll
+            for (int bx = 0; bx < C::kBoxes; ++bx) {
+              uint4* row = reinterpret_cast<uint4*>(smem + C::kSmemV + slot * C::kTileBytes + bx * C::kBoxBytes + r * 128);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) row[i] = make_uint4(0u, 0u, 0u, 0u);
+            }
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
         if (rescale && j > 0) {
           // the S tile arriving implies the previous P V has completed: O is stable
 #pragma unroll
@@ -553,12 +575,8 @@ moga_status launch(const Problem& p, cudaStream_t st) {
     return MOGA_ERR_CUDA;
   attn_schedule_kernel<<<1, 1024, 0, st>>>(p.grp, p.order, p.prefix, p.B, p.H);
   MOGA_CUDA_OK(cudaGetLastError());
-  static int num_sms = 0;
-  if (num_sms == 0) {
-    int dev = 0;
-    MOGA_CUDA_OK(cudaGetDevice(&dev));
-    MOGA_CUDA_OK(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
-  }
+  int num_sms = 0;
+  if (!current_sm_count(&num_sms)) return MOGA_ERR_CUDA;
   auto kern = attn_bf16_kernel<D>;
   MOGA_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::kDynSmem));
   const long long max_items = ((p.Tq + kQBlock - 1) / kQBlock + p.grp.G) * BH;
@@ -566,7 +584,8 @@ moga_status launch(const Problem& p, cudaStream_t st) {
   const float log2e = 1.4426950408889634f;
   kern<<<grid, kThreads, Cfg<D>::kDynSmem, st>>>(mq, mk, mv, p.grp, p.order, p.prefix,
                                                   static_cast<__nv_bfloat16*>(p.O), p.lse, p.header, (int)p.Tq,
-                                                  p.H, p.B * p.grp.G, p.scale * log2e, p.scale, p.sc);
+                                                  p.H, p.B * p.grp.G, p.scale * log2e, p.scale, p.sc,
+                                                  kDefaultWaitLimitNs);
   MOGA_CUDA_OK(cudaGetLastError());
   return MOGA_OK;
 }

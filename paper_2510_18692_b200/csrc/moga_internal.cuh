@@ -119,6 +119,14 @@ moga_status stga_build_host(int F, int Hh, int Ww, int wh, int ww, const int32_t
                             int tg, int augment, int32_t* q_idx, int32_t* q_inv, int32_t* q_offsets,
                             int32_t* kv_idx, int32_t* kv_offsets, int32_t* G_out, int32_t* Tkv_out);
 
+// Multiprocessor count of the current device (asked every time: a process may drive several
+// kinds of GPU, and the attribute query is a cached host-side lookup).
+inline bool current_sm_count(int* n) {
+  int dev = 0;
+  return cudaGetDevice(&dev) == cudaSuccess &&
+         cudaDeviceGetAttribute(n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && *n > 0;
+}
+
 #define MOGA_CUDA_OK(expr)                                   \
   do {                                                       \
     cudaError_t e__ = (expr);                                \

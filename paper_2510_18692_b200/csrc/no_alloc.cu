@@ -47,6 +47,15 @@ extern "C" moga_status moga_sort_static(const moga_shape* s, const int32_t* gid,
   const size_t need = moga_scratch_bytes(s);
   if (need == 0) return MOGA_ERR_UNSUPPORTED;
   auto ok = [](const void* p) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) & 15u) == 0; };
+  if (s->N == 0) {      // no tokens: every group is empty, as in moga_permute; no scratch is touched
+    if (!ok(offsets)) return MOGA_ERR_INVALID_ARG;
+    MOGA_CUDA_OK(cudaMemsetAsync(offsets, 0, sizeof(int32_t) * s->B * (s->M + 1), static_cast<cudaStream_t>(stream)));
+    if (status_out != nullptr) {
+      if (reinterpret_cast<uintptr_t>(status_out) & 7u) return MOGA_ERR_INVALID_ARG;
+      MOGA_CUDA_OK(cudaMemsetAsync(status_out, 0, 8, static_cast<cudaStream_t>(stream)));
+    }
+    return MOGA_OK;
+  }
   if (!ok(gid) || !ok(perm) || !ok(inv) || !ok(offsets) ||
       (status_out != nullptr && (reinterpret_cast<uintptr_t>(status_out) & 7u)))
     return MOGA_ERR_INVALID_ARG;

@@ -34,7 +34,6 @@ constexpr int kThreads = 192;
 constexpr int kTok = 128;                  // tokens per tile (MMA M)
 constexpr int kChunk = 64;                 // channels per stage: 128 bytes per row
 constexpr int kXBytes = kTok * 128;
-constexpr uint64_t kWaitLimitNs = 4000000000ull;
 
 template <int MP>
 struct RCfg {
@@ -76,7 +75,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 route_mma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW,
                  const float* __restrict__ bias, int32_t* __restrict__ gid, float* __restrict__ gate,
                  float* __restrict__ logits, uint32_t* header, long long total_tokens, int C, int M, int k,
-                 int gate_mode) {
+                 int gate_mode, uint64_t wait_limit_ns) {
   using R = RCfg<MP>;
   constexpr int NS = R::NS, NACC = R::NACC;
   extern __shared__ unsigned char smem_raw[];
@@ -111,22 +110,11 @@ route_mma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
   const uint32_t tmem = *tmem_slot;
 
   auto wait = [&](int idx, uint32_t parity, uint32_t where) -> bool {
-    const uint32_t b = bar(idx);
-    if (mbar_try_wait(b, parity)) return true;
-    const uint64_t t0 = global_timer_ns();
-    uint32_t spins = 0;
-    while (!mbar_try_wait(b, parity)) {
-      if ((++spins & 255u) == 0) {
-        if (*abort_flag) return false;
-        if (global_timer_ns() - t0 > kWaitLimitNs) {
-          *abort_flag = 1;
-          report_status(header, MOGA_ERR_TIMEOUT,
-                        (where << 24) | (1u << 23) | ((uint32_t)blockIdx.x << 8) | (uint32_t)idx);
-          return false;
-        }
-      }
-    }
-    return true;
+    const WaitResult res = mbar_wait_bounded(bar(idx), parity, abort_flag, wait_limit_ns);
+    if (res == kWaitExpired)
+      report_status(header, MOGA_ERR_TIMEOUT,
+                    (where << 24) | (1u << 23) | ((uint32_t)blockIdx.x << 8) | (uint32_t)idx);
+    return res == kWaitDone;
   };
 
   if (warp == 0) {
@@ -178,7 +166,6 @@ route_mma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
     const int q4 = warp & 3;                        // TMEM lane quarter this warp may read
     const int row = q4 * 32 + lane;
     const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16);
-    const int et = threadIdx.x - 64;                // 0..127 among the epilogue threads
     const int valid_cols = (nch < NACC ? nch : NACC) * R::kAccCols;
     uint32_t nt = 0;
     bool ok = true;
@@ -206,15 +193,10 @@ route_mma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
 #pragma unroll
       for (int i = 0; i < MP; ++i)
         if (i < M) ls[row * R::kLogitPitch + i] = r[i] + (bias != nullptr ? bias[i] : 0.f);
-      if (logits != nullptr) {
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        const long long tok0 = (long long)tile * kTok;
-        for (int idx = et; idx < kTok * M; idx += kTok) {
-          const int rr = idx / M, m = idx % M;
-          if (tok0 + rr < total_tokens) logits[(tok0 + rr) * M + m] = ls[rr * R::kLogitPitch + m];
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-      }
+      // optional output: each thread writes the row it owns, so no role ever waits on another
+      // outside the bounded mbarrier waits
+      if (logits != nullptr && tok < total_tokens)
+        for (int m = 0; m < M; ++m) logits[tok * M + m] = ls[row * R::kLogitPitch + m];
       if (tok < total_tokens)
         select_and_gate(ls + row * R::kLogitPitch, M, k, gate_mode, gid + tok * k, gate + tok * k);
     }
@@ -259,19 +241,15 @@ moga_status launch(const moga_shape& s, const WsLayout& L, const void* X, const 
   CUtensorMap mx, mw;
   if (!make_map_2d(&mx, X, total, s.C, kTok) || !make_map_2d(&mw, wsplit, 3 * MP, s.C, 3 * MP))
     return MOGA_ERR_CUDA;
-  static int num_sms = 0;
-  if (num_sms == 0) {
-    int dev = 0;
-    MOGA_CUDA_OK(cudaGetDevice(&dev));
-    MOGA_CUDA_OK(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
-  }
+  int num_sms = 0;
+  if (!current_sm_count(&num_sms)) return MOGA_ERR_CUDA;
   auto kern = route_mma_kernel<MP>;
   MOGA_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, R::kDynSmem));
   const long long ntiles = (total + kTok - 1) / kTok;
   const int grid = (int)(ntiles < num_sms ? ntiles : num_sms);
   kern<<<grid, kThreads, R::kDynSmem, st>>>(mx, mw, bias, gid, gate, logits,
                                             reinterpret_cast<uint32_t*>(ws + L.header), total, s.C, s.M, s.k,
-                                            s.gate_mode);
+                                            s.gate_mode, kDefaultWaitLimitNs);
   MOGA_CUDA_OK(cudaGetLastError());
   return MOGA_OK;
 }

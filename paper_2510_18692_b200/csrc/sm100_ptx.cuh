@@ -38,6 +38,28 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
+// Bounded wait on an mbarrier phase, the only way the tensor-core kernels wait.  It polls the
+// barrier; every 256 polls it looks at the CTA's abort flag (a shared-memory word another
+// role sets when its own wait ran out) and at the clock.  The caller reports kWaitExpired to
+// the host-visible status word and makes all roles leave; nothing here traps or spins forever.
+enum WaitResult : int { kWaitDone = 0, kWaitAborted = 1, kWaitExpired = 2 };
+constexpr uint64_t kDefaultWaitLimitNs = 4000000000ull;   // 4 s: far above any legitimate wait
+__device__ __forceinline__ WaitResult mbar_wait_bounded(uint32_t bar, uint32_t parity,
+                                                        volatile uint32_t* abort_flag, uint64_t limit_ns) {
+  if (mbar_try_wait(bar, parity)) return kWaitDone;
+  const uint64_t t0 = global_timer_ns();
+  uint32_t spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 255u) == 0) {
+      if (*abort_flag) return kWaitAborted;
+      if (global_timer_ns() - t0 > limit_ns) {
+        *abort_flag = 1;
+        return kWaitExpired;
+      }
+    }
+  }
+  return kWaitDone;
+}
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
                                             int c1, int c2) {
   asm volatile(

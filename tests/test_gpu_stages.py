@@ -255,6 +255,61 @@ def test_group_attn_peaky_bf16(mb):
     assert rel < 2e-2
 
 
+@pytest.mark.parametrize("dtype,D", [("bf16", 128), ("bf16", 64), ("f32", 64)])
+def test_group_attn_scale_zero_is_the_group_mean(mb, dtype, D):
+    """Closed form of Eq. 1: with scale = 0 every weight is 1 / n_g, so a row of the output is
+    the mean of its group's V rows.  Ragged sizes, so the tail tile's masked columns are met."""
+    sizes = [129, 300, 1, 0, 127, 513]
+    case = grouped_case(sizes, 2, D, dtype, seed=31, B=1)
+    cfg = _cfg(B=1, H=2, N=case["T"], D=D, M=len(sizes), k=1, dtype=dtype)
+    sh = mb.make_shape(cfg, scale=0.0)
+    Op = torch.full_like(case["Q"], float("nan"))
+    lse = torch.empty(1, 2, case["T"], dtype=torch.float32, device="cuda")
+    ws = mb.alloc_workspace(mb.moga_scratch_bytes(sh))
+    mb.moga_group_attn(sh, case["Q"], case["K"], case["V"], torch.from_numpy(case["offsets"]).cuda(), Op, lse, ws)
+    assert mb.moga_last_device_status(ws) == (0, 0)
+    V64 = case["V"].double().cpu().numpy()
+    want = np.zeros_like(V64)
+    off = case["offsets"][0]
+    for g in range(len(sizes)):
+        lo, hi = int(off[g]), int(off[g + 1])
+        if hi > lo:
+            want[:, :, lo:hi] = V64[:, :, lo:hi].mean(axis=2, keepdims=True)
+            assert (lse[:, :, lo:hi].double().cpu() - math.log(hi - lo)).abs().max().item() <= 1e-5
+    check_output(Op.float().cpu().numpy(), want, dtype, "Op at scale 0")
+    # and the oracle says the same (its own closed-form pin lives in the CPU tests)
+    ref = oracle.attn_all(to_np32(case["Q"]), to_np32(case["K"]), to_np32(case["V"]), case["gid"],
+                          np.ones((1, case["T"], 1)), case["offsets"], case["perm"], 0.0)
+    assert np.abs(ref - want).max() < 1e-12
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_group_attn_neighbour_group_values_do_not_leak(mb, dtype):
+    """Group independence (Eq. 5: keys and values of the token's own group only) must hold for
+    any stored values: the second group's K rows are huge and its V rows hold inf as data, and
+    the first group, whose tail tile shares a 128-row window with them, must come out
+    bit-identical to the run where the second group holds ordinary numbers."""
+    sizes = [200, 150]
+    case = grouped_case(sizes, 2, 128 if dtype == "bf16" else 64, dtype, seed=32, B=1)
+    D = case["Q"].shape[-1]
+    cfg = _cfg(B=1, H=2, N=case["T"], D=D, M=2, k=1, dtype=dtype)
+    sh = mb.make_shape(cfg, scale=1.0 / math.sqrt(D))
+    offsets = torch.from_numpy(case["offsets"]).cuda()
+    ws = mb.alloc_workspace(mb.moga_scratch_bytes(sh))
+    outs = []
+    for poison in (False, True):
+        K, V = case["K"].clone(), case["V"].clone()
+        if poison:
+            K[:, :, 200:] *= 1.0e30
+            V[:, :, 200:] = float("inf")
+        Op = torch.full_like(case["Q"], float("nan"))
+        mb.moga_group_attn(sh, case["Q"], K, V, offsets, Op, None, ws)
+        assert mb.moga_last_device_status(ws) == (0, 0)
+        outs.append(Op[:, :, :200].clone())
+    assert torch.isfinite(outs[1].float()).all()
+    assert torch.equal(outs[0], outs[1])
+
+
 @pytest.mark.parametrize("grow", [3.0, 24.0])
 def test_group_attn_growing_scores_bf16(mb, grow):
     """Keys late in each group are scaled up, so later K/V tiles hold scores far above the

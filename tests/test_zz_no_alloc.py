@@ -3,11 +3,13 @@ they need it (their framework's pool owns the GPU, or their budget was fixed at
 start-up).  Its scratch is a device array inside the library, so the test checks that
 two calls in a row -- which share that array and find the previous call's words in
 it -- each give exactly what the workspace entry point (moga_permute, indices only)
-gives.  Integer outputs: the comparison is bit for bit.  Collected last on purpose."""
+gives, and exactly what the CPU oracle's sort of the same assignments gives.  Integer
+outputs: the comparisons are bit for bit.  Collected last on purpose."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2510_18692_b200.inputs import GATE_SOFTMAX_ALL, MogaConfig
 
 pytestmark = pytest.mark.gpu
@@ -46,6 +48,10 @@ def test_static_sort_matches_workspace_sort_twice_in_a_row():
         for a, b in zip(ref, got):
             assert torch.equal(a, b)
         assert status.tolist() == [0, 0]
+        o_off, o_perm, o_inv = oracle.sort(gid.cpu().numpy(), M)
+        assert np.array_equal(got[0].cpu().numpy(), o_perm)
+        assert np.array_equal(got[1].cpu().numpy(), o_inv)
+        assert np.array_equal(got[2].cpu().numpy(), o_off)
     # a bad group id is clamped and reported through status_out, like the workspace variant
     gid[0, 5, 0] = 99
     mb.moga_sort_static(sh, gid, got[0], got[1], got[2], status)
@@ -56,6 +62,17 @@ def test_static_sort_matches_workspace_sort_twice_in_a_row():
     mb.moga_sort_static(sh, gid, got[0], got[1], got[2], status)
     torch.cuda.synchronize()
     assert status.tolist() == [0, 0]
+
+
+def test_static_sort_of_no_tokens_is_a_no_op_with_zero_offsets():
+    from paper_2510_18692_b200 import binding as mb
+    cfg = MogaConfig("empty", 2, 1, 0, 64, 64, 8, 1, "bf16", GATE_SOFTMAX_ALL, 0)
+    sh = mb.make_shape(cfg)
+    offsets = torch.full((2, 9), 5, dtype=torch.int32, device="cuda")
+    status = torch.full((2,), 77, dtype=torch.int32, device="cuda")
+    mb.moga_sort_static(sh, None, None, None, offsets, status)
+    torch.cuda.synchronize()
+    assert not offsets.any() and status.tolist() == [0, 0]
 
 
 def test_static_sort_rejects_what_does_not_fit():
