@@ -164,6 +164,11 @@ moga_status moga_sort_static(const moga_shape* s, const int32_t* gid, int32_t* p
  * boundary.  bf16 runs on tcgen05 tensor cores (fp32 accumulate and softmax);
  * fp32 runs on the fp32 ALUs.  lse may be NULL.  ws: at least moga_scratch_bytes.
  * An empty group does no work; a 1-token group returns its own V row.
+ * scale = 0 gives uniform weights (the group mean of V).  Groups are independent for any K:
+ * scores against rows of a neighbouring group that share a 128-key tile are masked before they
+ * are used.  The bf16 kernel does load such neighbouring V rows and multiplies them by an
+ * exact-zero weight, so V must be finite (0 x inf is NaN): a non-finite V row can reach the
+ * rows of the group stored just before it.  The fp32 kernel never loads a foreign row.
  */
 moga_status moga_group_attn(const moga_shape* s, const void* Qp, const void* Kp, const void* Vp,
                             const int32_t* offsets, void* Op, float* lse, void* ws,

@@ -25,8 +25,6 @@
 #include "moga_internal.cuh"
 #include "sm100_ptx.cuh"
 
-#include <type_traits>
-
 namespace moga {
 namespace {
 
@@ -154,7 +152,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                  const __grid_constant__ CUtensorMap mapV, const Groups grp,
                  const int32_t* __restrict__ order, const int32_t* __restrict__ prefix,
                  __nv_bfloat16* __restrict__ Op, float* __restrict__ lse, uint32_t* header, int T, int H,
-                 int BG, float scale_log2, float scale, const Scatter sc, uint64_t wait_limit_ns) {
+                 int BG, float scale_log2, float scale, const Scatter sc) {
   using C = Cfg<D>;
   constexpr int NS = C::NS;
   extern __shared__ unsigned char smem_raw[];
@@ -206,7 +204,16 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 
   // Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
   auto wait = [&](int idx, uint32_t parity, uint32_t where) -> bool {
-    const WaitResult res = mbar_wait_bounded(bar(idx), parity, abort_flag, wait_limit_ns);
+    const WaitResult res = mbar_wait_bounded(bar(idx), parity, abort_flag, kDefaultWaitLimitNs);
+    if (res == kWaitExpired)
+      report_status(header, MOGA_ERR_TIMEOUT, (where << 24) | ((uint32_t)blockIdx.x << 8) | (uint32_t)idx);
+    return res == kWaitDone;
+  };
+
+  // The producer's waits are long (a ring slot frees once per K/V tile): it parks between polls
+  // so that it does not take issue slots from the softmax warps of its sub-partition.
+  auto wait_parked = [&](int idx, uint32_t parity, uint32_t where) -> bool {
+    const WaitResult res = mbar_wait_bounded_parked(bar(idx), parity, abort_flag, kDefaultWaitLimitNs);
     if (res == kWaitExpired)
       report_status(header, MOGA_ERR_TIMEOUT, (where << 24) | ((uint32_t)blockIdx.x << 8) | (uint32_t)idx);
     return res == kWaitDone;
@@ -217,6 +224,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
   // (each setmaxnreg sits at the top of the branch it governs, so the compiler can give
   //  the code it dominates that many registers)
   if (warp < 4) {
+    static_assert(128 * 80 + 256 * 208 <= kThreads * 168, "the softmax warps' setmaxnreg.inc would wait forever");
     reg_dec<80>();
   if (warp == 0) {
     // ===================================================================== TMA producer
@@ -228,7 +236,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         const int ntiles = (it.khi - it.klo + kTileN - 1) / kTileN;
         const bool validB = it.row0 + kTileM < it.qhi;
         for (int x = 0; x < (validB ? 2 : 1) && ok; ++x) {
-          ok = wait(Q_EMPTY + x, (nq[x] & 1u) ^ 1u, 1);
+          ok = wait_parked(Q_EMPTY + x, (nq[x] & 1u) ^ 1u, 1);
           if (!ok) break;
           mbar_expect_tx(bar(Q_FULL + x), C::kTileBytes);
 #pragma unroll
@@ -240,14 +248,14 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         for (int j = 0; j < ntiles && ok; ++j) {
           const int s = nkv % NS;
           const uint32_t ph = ((nkv / NS) & 1u) ^ 1u;
-          ok = wait(K_EMPTY + s, ph, 2);
+          ok = wait_parked(K_EMPTY + s, ph, 2);
           if (!ok) break;
           mbar_expect_tx(bar(K_FULL + s), C::kTileBytes);
 #pragma unroll
           for (int bx = 0; bx < C::kBoxes; ++bx)
             tma_load_3d(sK + s * C::kTileBytes + bx * C::kBoxBytes, &mapK, bar(K_FULL + s), bx * 64,
                         it.klo + j * kTileN, it.bh);
-          ok = wait(V_EMPTY + s, ph, 3);
+          ok = wait_parked(V_EMPTY + s, ph, 3);
           if (!ok) break;
           mbar_expect_tx(bar(V_FULL + s), C::kTileBytes);
 #pragma unroll
@@ -311,6 +319,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             ok = wait(K_FULL + nk % NS, (nk / NS) & 1u, 7);
             if (!ok) break;
           }
+          // ragged last tile, landed: warp 2 clears its foreign V rows while the softmax runs
           for (int x = 0; x < nx && ok; ++x) {
             ok = wait(P_FULL + x, np[x] & 1u, 8);
             if (!ok) break;
@@ -351,14 +360,12 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     const uint32_t tS = tmem + lane_off + x * kTileN;
     const uint32_t tO = tmem + lane_off + 256 + x * 128;
-    uint32_t n_s = 0, n_o = 0, n_kv = 0;             // n_kv: K/V tiles of earlier items (ring position)
+    uint32_t n_s = 0, n_o = 0;
     bool ok = true;
     for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
       const Item it = decode_item(w, grp, order, prefix, BG, H);
-      const int ntiles = (it.khi - it.klo + kTileN - 1) / kTileN;
-      const uint32_t kv0 = n_kv;
-      n_kv += (uint32_t)ntiles;
       if (x == 1 && !(it.row0 + kTileM < it.qhi)) continue;
+      const int ntiles = (it.khi - it.klo + kTileN - 1) / kTileN;
       const int tile_row0 = it.row0 + x * kTileM;
       float m = -INFINITY, l = 0.f;
       for (int j = 0; j < ntiles && ok; ++j) {
@@ -380,10 +387,11 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 #pragma unroll
           for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[c * 32]));
           tmem_wait_ld();
-          const bool ragged = ncols < kTileN;
-          if (ragged && exact) {
-            // columns past the group's last key hold scores against the next group's rows:
-            // keep them out of the maximum (comparisons only, so scale = 0 cannot make a NaN)
+          if (ncols < kTileN) {
+            // Columns past the group's last key hold scores against the next group's rows (any
+            // value, NaN included): they become -inf before anything reads them, so they never
+            // win the maximum and their weight is 2^(-inf) = 0 exactly.  (scale_log2 > 0 always:
+            // the launcher replaces a zero scale by the smallest normal float, see there.)
 #pragma unroll
             for (int c = 0; c < 128; ++c)
               if (c >= ncols) sreg[c] = 0xff800000u;        // -inf
@@ -404,24 +412,15 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
           const float neg_m = -m * scale_log2;
           const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(neg_m, neg_m);
           float2 ls[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
-          // p = 2^(s * scale_log2 - m * scale_log2); on a ragged tile the weight of a column past
-          // the last key is an exact 0 selected after the exponential, whatever its score holds
-          auto weights = [&](auto masked) {
 #pragma unroll
-            for (int c = 0; c < 64; ++c) {
-              const float2 x = __ffma2_rn(make_float2(__uint_as_float(sreg[2 * c]), __uint_as_float(sreg[2 * c + 1])),
-                                          sc2, nm2);
-              float2 pe = make_float2(ex2(x.x), ex2(x.y));
-              if (decltype(masked)::value) {
-                pe.x = 2 * c < ncols ? pe.x : 0.f;
-                pe.y = 2 * c + 1 < ncols ? pe.y : 0.f;
-              }
-              ls[c & 3] = __fadd2_rn(ls[c & 3], pe);
-              __nv_bfloat162 pk = __floats2bfloat162_rn(pe.x, pe.y);
-              preg[c] = *reinterpret_cast<uint32_t*>(&pk);
-            }
-          };
-          if (ragged) weights(std::true_type{}); else weights(std::false_type{});
+          for (int c = 0; c < 64; ++c) {
+            const float2 x = __ffma2_rn(make_float2(__uint_as_float(sreg[2 * c]), __uint_as_float(sreg[2 * c + 1])),
+                                        sc2, nm2);
+            const float2 pe = make_float2(ex2(x.x), ex2(x.y));
+            ls[c & 3] = __fadd2_rn(ls[c & 3], pe);
+            __nv_bfloat162 pk = __floats2bfloat162_rn(pe.x, pe.y);
+            preg[c] = *reinterpret_cast<uint32_t*>(&pk);
+          }
           const float2 l01 = __fadd2_rn(__fadd2_rn(ls[0], ls[1]), __fadd2_rn(ls[2], ls[3]));
           lsum = l01.x + l01.y;
           if (exact || !__any_sync(0xffffffffu, !(lsum < kRowSumLimit))) break;
@@ -430,24 +429,6 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         l = l * alpha + lsum;
         tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&preg[0]));
         tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&preg[32]));
-        if (x == 0 && ncols < kTileN) {
-          // Ragged last tile: the V rows past the group's last key belong to the next group (or
-          // are the zero fill past T).  Their weights are 0, but 0 x inf would still poison O, so
-          // tile A's warps clear those rows in shared memory before either tile's P V is issued
-          // (the MMA warp waits for P_FULL of tile A first).  Thread r owns key row r.
-          const uint32_t slot = (kv0 + (uint32_t)j) % NS;
-          ok = __all_sync(0xffffffffu, wait(V_FULL + slot, ((kv0 + (uint32_t)j) / NS) & 1u, 12));
-          if (!ok) break;
-          if (r >= ncols) {
-#pragma unroll
-            for (int bx = 0; bx < C::kBoxes; ++bx) {
-              uint4* row = reinterpret_cast<uint4*>(smem + C::kSmemV + slot * C::kTileBytes + bx * C::kBoxBytes + r * 128);
-#pragma unroll
-              for (int i = 0; i < 8; ++i) row[i] = make_uint4(0u, 0u, 0u, 0u);
-            }
-          }
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        }
         if (rescale && j > 0) {
           // the S tile arriving implies the previous P V has completed: O is stable
 #pragma unroll
@@ -581,11 +562,15 @@ moga_status launch(const Problem& p, cudaStream_t st) {
   MOGA_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::kDynSmem));
   const long long max_items = ((p.Tq + kQBlock - 1) / kQBlock + p.grp.G) * BH;
   const int grid = (int)(max_items < num_sms ? max_items : num_sms);
+  // The kernel works in the log2 domain with scale_log2 = scale * log2(e) and masks columns by
+  // setting their score to -inf, which needs scale_log2 > 0 (-inf * 0 is NaN).  A zero scale
+  // (uniform weights) is served by the smallest normal float instead: every weight
+  // 2^(1.2e-38 * (s - m)) is then exactly 1.0f for all scores below 1e30 in magnitude.
   const float log2e = 1.4426950408889634f;
+  const float scale_log2 = p.scale * log2e > 1.17549435e-38f ? p.scale * log2e : 1.17549435e-38f;
   kern<<<grid, kThreads, Cfg<D>::kDynSmem, st>>>(mq, mk, mv, p.grp, p.order, p.prefix,
                                                   static_cast<__nv_bfloat16*>(p.O), p.lse, p.header, (int)p.Tq,
-                                                  p.H, p.B * p.grp.G, p.scale * log2e, p.scale, p.sc,
-                                                  kDefaultWaitLimitNs);
+                                                  p.H, p.B * p.grp.G, scale_log2, p.scale, p.sc);
   MOGA_CUDA_OK(cudaGetLastError());
   return MOGA_OK;
 }

@@ -33,6 +33,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// try_wait with a suspend-time hint: the hardware may park the thread until the phase
+// completes or `hint_ns` have passed, so a role that waits long does not compete for issue slots.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ uint64_t global_timer_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -56,6 +69,22 @@ __device__ __forceinline__ WaitResult mbar_wait_bounded(uint32_t bar, uint32_t p
         *abort_flag = 1;
         return kWaitExpired;
       }
+    }
+  }
+  return kWaitDone;
+}
+// The same bounded wait for a role that expects to wait long (microseconds or more): each
+// poll parks the thread for up to kParkNs, then the abort flag and the clock are looked at.
+constexpr uint32_t kParkNs = 20000;
+__device__ __forceinline__ WaitResult mbar_wait_bounded_parked(uint32_t bar, uint32_t parity,
+                                                               volatile uint32_t* abort_flag, uint64_t limit_ns) {
+  if (mbar_try_wait(bar, parity)) return kWaitDone;
+  const uint64_t t0 = global_timer_ns();
+  while (!mbar_try_wait_hint(bar, parity, kParkNs)) {
+    if (*abort_flag) return kWaitAborted;
+    if (global_timer_ns() - t0 > limit_ns) {
+      *abort_flag = 1;
+      return kWaitExpired;
     }
   }
   return kWaitDone;
