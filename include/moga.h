@@ -308,6 +308,19 @@ moga_status moga_forward_host(const moga_shape* s, const void* X, const float* W
 moga_status moga_last_device_status(void* ws, void* stream, uint32_t* detail);
 
 /*
+ * Choice of the bf16 group-attention kernel (the paper has no counterpart: a tuning and test
+ * switch).  Two kernels compute Eq. 1 inside the groups on the tensor cores: one gives a block
+ * of 256 query rows to one SM; the other gives 512 query rows to a pair of SMs that share every
+ * K/V tile (each SM stages half of it), for d_head = 128.  MOGA_ATTN_AUTO picks the pair kernel
+ * when the launch's groups are long (>= 2,048 query rows per group on average) and the one-SM
+ * kernel otherwise; the other two values force one of them (the pair kernel still needs
+ * d_head = 128, else the one-SM kernel runs).  Process-wide, not thread-safe against
+ * concurrent launches; returns MOGA_ERR_INVALID_ARG for another value.
+ */
+typedef enum { MOGA_ATTN_AUTO = 0, MOGA_ATTN_SINGLE = 1, MOGA_ATTN_PAIR = 2 } moga_attn_kernel;
+moga_status moga_set_attn_kernel(int32_t mode);
+
+/*
  * Self-test of the time-out path (the paper has no counterpart: it is a diagnostic).
  * Every wait inside the tensor-core kernels is bounded; when one runs out the kernel writes
  * MOGA_ERR_TIMEOUT and a detail word to the status header and returns normally.  This call

@@ -22,40 +22,14 @@
 // P (bf16, two per column) overwrites the first 64 columns of its S tile.
 // Every mbarrier wait is bounded: on expiry the CTA records MOGA_ERR_TIMEOUT in the
 // workspace status word, all roles leave their loops, and TMEM is released.
-#include "moga_internal.cuh"
-#include "sm100_ptx.cuh"
+#include "attn_common.cuh"
 
 namespace moga {
-namespace {
-
-constexpr int kThreads = 384;
-constexpr int kTileM = 128;       // query rows per tile
-constexpr int kTileN = 128;       // keys per K/V tile
-constexpr int kQBlock = 2 * kTileM;
-constexpr float kRowSumLimit = 1.0995116e12f;      // 2^40: a tile's row sum beyond this forces a new maximum
-
-using namespace sm100;
+namespace attn {
 
 // ----------------------------------------------------------------------------- schedule
-// The groups of one launch.  Group g of batch item b owns query rows
-// [q_off[b*stride + g], q_off[b*stride + g + 1]) of Q / O and key rows
-// [kv_off[b*stride + g], kv_off[b*stride + g + 1]) of K / V.  Routed groups (Alg. 1): q_off and
-// kv_off are the same array, stride = G + 1.  Static groups (Sec. 3.2): one list shared by
-// all batch items (stride 0), keys may be a superset of the queries.
-struct Groups {
-  const int32_t* q_off;
-  const int32_t* kv_off;
-  int stride;
-  int G;
-};
-
-constexpr int kRankLimit = 256;   // above this many groups per item the list keeps its order
-
-// order[b*G + r]  : group with the r-th largest cost (queries x keys) in batch item b
-// prefix[b*G + r] : number of work items before (b, r); prefix[B*G] = total
-// A group with queries but no keys gets no work item: its rows are left untouched.
 __global__ void attn_schedule_kernel(const Groups grp, int32_t* __restrict__ order, int32_t* __restrict__ prefix,
-                                     int B, int H) {
+                                     int B, int H, int qblock) {
   const int G = grp.G;
   for (int idx = threadIdx.x; idx < B * G; idx += blockDim.x) {
     const int b = idx / G, g = idx % G;
@@ -81,42 +55,25 @@ __global__ void attn_schedule_kernel(const Groups grp, int32_t* __restrict__ ord
       const int nq = grp.q_off[(size_t)b * grp.stride + g + 1] - grp.q_off[(size_t)b * grp.stride + g];
       const int nk = grp.kv_off[(size_t)b * grp.stride + g + 1] - grp.kv_off[(size_t)b * grp.stride + g];
       prefix[idx] = acc;
-      if (nk > 0) acc += ((nq + kQBlock - 1) / kQBlock) * H;
+      if (nk > 0) acc += ((nq + qblock - 1) / qblock) * H;
     }
     prefix[B * G] = acc;
   }
 }
 
-struct Item {
-  int bh;          // b * H + h
-  int row0;        // first row of the query block
-  int qhi;         // end of the group's query rows
-  int klo, khi;    // the group's key rows
-};
+}  // namespace attn
 
-__device__ __forceinline__ Item decode_item(int w, const Groups& grp, const int32_t* __restrict__ order,
-                                            const int32_t* __restrict__ prefix, int BG, int H) {
-  int lo = 0, hi = BG;           // largest idx with prefix[idx] <= w (entries without items are skipped)
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if (prefix[mid] <= w) lo = mid; else hi = mid;
-  }
-  const int b = lo / grp.G;
-  const int g = order[lo];
-  const int32_t* qo = grp.q_off + (size_t)b * grp.stride;
-  const int32_t* ko = grp.kv_off + (size_t)b * grp.stride;
-  Item it;
-  const int qlo = qo[g];
-  it.qhi = qo[g + 1];
-  it.klo = ko[g];
-  it.khi = ko[g + 1];
-  const int nqb = (it.qhi - qlo + kQBlock - 1) / kQBlock;
-  const int local = w - prefix[lo];
-  const int h = local / nqb, qb = local % nqb;
-  it.bh = b * H + h;
-  it.row0 = qlo + qb * kQBlock;
-  return it;
-}
+namespace {
+
+using namespace attn;
+
+constexpr int kThreads = 384;
+constexpr int kTileM = 128;       // query rows per tile
+constexpr int kTileN = 128;       // keys per K/V tile
+constexpr int kQBlock = 2 * kTileM;
+constexpr float kRowSumLimit = 1.0995116e12f;      // 2^40: a tile's row sum beyond this forces a new maximum
+
+using namespace sm100;
 
 // ----------------------------------------------------------------------------- the kernel
 template <int D>
@@ -133,17 +90,6 @@ struct Cfg {
   static constexpr int kNumBars = 2 + 2 + 4 * NS + 2 + 2 + 2 + 2;
   static constexpr int kSmemTotal = kSmemBar + 8 * kNumBars + 16;
   static constexpr int kDynSmem = kSmemTotal + 1024;      // slack for 1024-byte alignment
-};
-
-// Output placement.  perm == nullptr: rows stay in sorted order, Op is [B*H, T, D].
-// Otherwise (top-1 routing) the epilogue is the gated inverse permutation of Eq. 5: sorted
-// row p of batch item b goes to token perm[b, p] of O (element strides sb, sh, sn),
-// multiplied by gate[b, token] in fp32 before the one rounding to bf16.
-struct Scatter {
-  const int32_t* perm;
-  const float* gate;
-  long long sb, sh, sn;
-  int N;
 };
 
 template <int D>
@@ -232,7 +178,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       uint32_t nq[2] = {0, 0}, nkv = 0;
       bool ok = true;
       for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
-        const Item it = decode_item(w, grp, order, prefix, BG, H);
+        const Item it = decode_item<kQBlock>(w, grp, order, prefix, BG, H);
         const int ntiles = (it.khi - it.klo + kTileN - 1) / kTileN;
         const bool validB = it.row0 + kTileM < it.qhi;
         for (int x = 0; x < (validB ? 2 : 1) && ok; ++x) {
@@ -292,7 +238,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                  (accumulate || kk > 0) ? 1u : 0u);
       };
       for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
-        const Item it = decode_item(w, grp, order, prefix, BG, H);
+        const Item it = decode_item<kQBlock>(w, grp, order, prefix, BG, H);
         const int ntiles = (it.khi - it.klo + kTileN - 1) / kTileN;
         const int nx = (it.row0 + kTileM < it.qhi) ? 2 : 1;
         // first S tiles
@@ -363,7 +309,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     uint32_t n_s = 0, n_o = 0;
     bool ok = true;
     for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
-      const Item it = decode_item(w, grp, order, prefix, BG, H);
+      const Item it = decode_item<kQBlock>(w, grp, order, prefix, BG, H);
       if (x == 1 && !(it.row0 + kTileM < it.qhi)) continue;
       const int ntiles = (it.khi - it.klo + kTileN - 1) / kTileN;
       const int tile_row0 = it.row0 + x * kTileM;
@@ -521,40 +467,14 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 }
 
 // ----------------------------------------------------------------------------- host side
-// [B*H, T, D] bf16, box 64 x 128 x 1, 128-byte swizzle, out-of-range rows read as zero.
-bool make_map(CUtensorMap* map, const void* ptr, int D, long long T, long long BH) {
-  EncodeTiledFn fn = get_encode_fn();
-  if (fn == nullptr) return false;
-  cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)T, (cuuint64_t)BH};
-  cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)T * D * 2};
-  cuuint32_t box[3] = {64, (cuuint32_t)kTileM, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// One launch: B*H heads, groups grp, Q / O with Tq rows and K / V with Tkv rows per head.
-struct Problem {
-  int B, H;
-  long long Tq, Tkv;
-  float scale;
-  const void *Q, *K, *V;
-  void* O;
-  float* lse;
-  Groups grp;
-  int32_t *order, *prefix;   // scratch: B*G and B*G + 1 int32
-  uint32_t* header;          // device status word
-  Scatter sc;
-};
-
 template <int D>
-moga_status launch(const Problem& p, cudaStream_t st) {
+moga_status launch_one(const Problem& p, cudaStream_t st) {
   CUtensorMap mq, mk, mv;
   const long long BH = (long long)p.B * p.H;
-  if (!make_map(&mq, p.Q, D, p.Tq, BH) || !make_map(&mk, p.K, D, p.Tkv, BH) || !make_map(&mv, p.V, D, p.Tkv, BH))
+  if (!make_map(&mq, p.Q, D, p.Tq, BH, kTileM) || !make_map(&mk, p.K, D, p.Tkv, BH, kTileN) ||
+      !make_map(&mv, p.V, D, p.Tkv, BH, kTileN))
     return MOGA_ERR_CUDA;
-  attn_schedule_kernel<<<1, 1024, 0, st>>>(p.grp, p.order, p.prefix, p.B, p.H);
+  attn_schedule_kernel<<<1, 1024, 0, st>>>(p.grp, p.order, p.prefix, p.B, p.H, kQBlock);
   MOGA_CUDA_OK(cudaGetLastError());
   int num_sms = 0;
   if (!current_sm_count(&num_sms)) return MOGA_ERR_CUDA;
@@ -575,8 +495,18 @@ moga_status launch(const Problem& p, cudaStream_t st) {
   return MOGA_OK;
 }
 
+// Which kernel serves a launch.  The CTA-pair kernel (D = 128 only) halves the K/V bytes each
+// SM stages and reads per flop, but its work item is 512 query rows: it takes the launches whose
+// groups are long (mean of at least kPairMinRows query rows per group); short groups, such as
+// the static ones of Sec. 3.2, and D = 64 stay on the one-CTA kernel.  g_attn_kernel overrides
+// the choice (moga_set_attn_kernel).
+constexpr long long kPairMinRows = 2048;
+int g_attn_kernel = MOGA_ATTN_AUTO;
+
 moga_status launch_any(int D, const Problem& p, cudaStream_t st) {
-  return D == 128 ? launch<128>(p, st) : launch<64>(p, st);
+  const bool long_groups = p.grp.G > 0 && p.Tq / p.grp.G >= kPairMinRows;
+  const bool pair = D == 128 && (g_attn_kernel == MOGA_ATTN_PAIR || (g_attn_kernel == MOGA_ATTN_AUTO && long_groups));
+  return pair ? launch_pair(p, st) : launch_single(D, p, st);
 }
 
 // Routed groups: offsets [B, M+1] serve queries and keys alike; scratch from the workspace layout.
@@ -589,6 +519,12 @@ Problem routed_problem(const moga_shape& s, const WsLayout& L, const void* Qp, c
 }
 
 }  // namespace
+
+moga_status attn::launch_single(int D, const attn::Problem& p, cudaStream_t st) {
+  return D == 128 ? launch_one<128>(p, st) : launch_one<64>(p, st);
+}
+
+void set_attn_kernel(int mode) { g_attn_kernel = mode; }
 
 moga_status launch_attn_bf16(const moga_shape& s, const WsLayout& L, const void* Qp, const void* Kp,
                              const void* Vp, const int32_t* offsets, void* Op, float* lse, char* ws,

@@ -351,6 +351,12 @@ moga_status moga_visual_forward(const moga_shape* s, const void* X, const float*
   return launch_mean3(*s, w + v.A, w + v.Bs, lists->q_inv, w + v.C, O, cs);
 }
 
+moga_status moga_set_attn_kernel(int32_t mode) {
+  if (mode != MOGA_ATTN_AUTO && mode != MOGA_ATTN_SINGLE && mode != MOGA_ATTN_PAIR) return MOGA_ERR_INVALID_ARG;
+  set_attn_kernel(mode);
+  return MOGA_OK;
+}
+
 moga_status moga_last_device_status(void* ws, void* stream, uint32_t* detail) {
   if (ws == nullptr) return MOGA_ERR_WORKSPACE;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);

@@ -110,6 +110,7 @@ moga_status launch_attn_f32_groups(int B, int H, int D, float scale, int G, int 
                                    const float* Kp, const float* Vp, const int32_t* q_offsets,
                                    const int32_t* kv_offsets, int off_stride, float* Op, float* lse,
                                    cudaStream_t st);
+void set_attn_kernel(int mode);
 moga_status launch_gather_list(const moga_shape& s, const int32_t* idx, int L, const void* src, void* dst,
                                cudaStream_t st);
 moga_status launch_frame_offsets(int32_t* off, int F, int tokens_per_frame, cudaStream_t st);

@@ -237,6 +237,50 @@ def test_group_attn(mb, dtype, D, sizes):
             assert (lse[:, :, lo:hi].double().cpu() - ref).abs().max().item() <= (1e-4 if dtype == "f32" else 2e-2)
 
 
+PAIR_SIZES = [
+    [512, 300, 129, 128, 127, 1, 0, 2, 65, 0, 1000],
+    [1], [0, 0, 3], [257], [513], [4096], [1500, 2600, 640],
+]
+
+
+@pytest.mark.parametrize("sizes", PAIR_SIZES, ids=lambda s: "g" + "_".join(map(str, s[:4])))
+def test_group_attn_pair_kernel(mb, sizes):
+    """The CTA-pair kernel (512 query rows per pair of SMs, d_head = 128), forced for every group
+    size, against the oracle and against the one-CTA kernel; then the automatic choice."""
+    H, B, D = 2, 2, 128
+    case = grouped_case(sizes, H, D, "bf16", seed=len(sizes) + 7, B=B)
+    T, M = case["T"], len(sizes)
+    cfg = _cfg(B=B, H=H, N=T, D=D, M=M, k=1, dtype="bf16")
+    scale = 1.0 / math.sqrt(D)
+    sh = mb.make_shape(cfg, scale=scale)
+    offsets = torch.from_numpy(case["offsets"]).cuda()
+    ws = mb.alloc_workspace(mb.moga_scratch_bytes(sh))
+    want = oracle.attn_all(to_np32(case["Q"]), to_np32(case["K"]), to_np32(case["V"]), case["gid"],
+                           np.ones((B, T, 1)), case["offsets"], case["perm"], scale)
+    outs = {}
+    try:
+        for mode in (mb.MOGA_ATTN_PAIR, mb.MOGA_ATTN_SINGLE):
+            mb.moga_set_attn_kernel(mode)
+            Op = torch.full_like(case["Q"], float("nan"))
+            lse = torch.empty(B, H, T, dtype=torch.float32, device="cuda")
+            mb.moga_group_attn(sh, case["Q"], case["K"], case["V"], offsets, Op, lse, ws)
+            assert mb.moga_last_device_status(ws) == (0, 0)
+            check_output(Op.float().cpu().numpy(), want, "bf16", f"Op (kernel {mode})")
+            outs[mode] = (Op, lse)
+    finally:
+        mb.moga_set_attn_kernel(mb.MOGA_ATTN_AUTO)
+    # same arithmetic per row in both kernels: expected equal to the last bit; at the least very close
+    a, b = outs[mb.MOGA_ATTN_PAIR], outs[mb.MOGA_ATTN_SINGLE]
+    assert (a[0].float() - b[0].float()).abs().max().item() <= 2.0 ** -7 * b[0].float().abs().max().item() + 1e-6
+    assert (a[1] - b[1]).abs().max().item() <= 1e-3
+    q, k_ = case["Q"].double().cpu(), case["K"].double().cpu()
+    for g in range(M):
+        lo, hi = case["offsets"][0, g], case["offsets"][0, g + 1]
+        if hi > lo:
+            ref = torch.logsumexp(torch.einsum("bhnd,bhmd->bhnm", q[:, :, lo:hi], k_[:, :, lo:hi]) * scale, -1)
+            assert (a[1][:, :, lo:hi].double().cpu() - ref).abs().max().item() <= 2e-2
+
+
 def test_group_attn_peaky_bf16(mb):
     """Large score spread (Q scaled x4): exercises the running-max rescale."""
     case = grouped_case([700, 333], 2, 128, "bf16", seed=9, B=1, qscale=4.0)
