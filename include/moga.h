@@ -309,13 +309,14 @@ moga_status moga_last_device_status(void* ws, void* stream, uint32_t* detail);
 
 /*
  * Choice of the bf16 group-attention kernel (the paper has no counterpart: a tuning and test
- * switch).  Two kernels compute Eq. 1 inside the groups on the tensor cores: one gives a block
- * of 256 query rows to one SM; the other gives 512 query rows to a pair of SMs that share every
- * K/V tile (each SM stages half of it), for d_head = 128.  MOGA_ATTN_AUTO picks the pair kernel
- * when the launch's groups are long (>= 2,048 query rows per group on average) and the one-SM
- * kernel otherwise; the other two values force one of them (the pair kernel still needs
- * d_head = 128, else the one-SM kernel runs).  Process-wide, not thread-safe against
- * concurrent launches; returns MOGA_ERR_INVALID_ARG for another value.
+ * switch).  Two kernels compute Eq. 1 inside the groups on the tensor cores.  The default
+ * (MOGA_ATTN_AUTO, same as MOGA_ATTN_SINGLE) gives a block of 256 query rows to one SM.
+ * MOGA_ATTN_PAIR gives 256 query rows to a pair of SMs that issue every tensor-core
+ * instruction together and each stage half of every K/V tile (d_head = 128, routed launches
+ * only; other launches keep the default).  The pair kernel is correct on every shape but
+ * measured slower (see the kernel selection comment in csrc/attn_bf16.cu); it is kept as an
+ * option.  Process-wide, not thread-safe against concurrent launches; returns
+ * MOGA_ERR_INVALID_ARG for another value.
  */
 typedef enum { MOGA_ATTN_AUTO = 0, MOGA_ATTN_SINGLE = 1, MOGA_ATTN_PAIR = 2 } moga_attn_kernel;
 moga_status moga_set_attn_kernel(int32_t mode);

@@ -92,13 +92,14 @@ struct Cfg {
   static constexpr int kDynSmem = kSmemTotal + 1024;      // slack for 1024-byte alignment
 };
 
-template <int D>
+// Redo: the work items are those listed in redo[4 ...] (redo[0] of them) instead of all items.
+template <int D, bool Redo>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                  const __grid_constant__ CUtensorMap mapV, const Groups grp,
                  const int32_t* __restrict__ order, const int32_t* __restrict__ prefix,
                  __nv_bfloat16* __restrict__ Op, float* __restrict__ lse, uint32_t* header, int T, int H,
-                 int BG, float scale_log2, float scale, const Scatter sc) {
+                 int BG, float scale_log2, float scale, const Scatter sc, const int32_t* __restrict__ redo) {
   using C = Cfg<D>;
   constexpr int NS = C::NS;
   extern __shared__ unsigned char smem_raw[];
@@ -115,7 +116,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total_items = prefix[BG];
+  const int total_items = Redo ? redo[0] : prefix[BG];
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
@@ -178,7 +179,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       uint32_t nq[2] = {0, 0}, nkv = 0;
       bool ok = true;
       for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
-        const Item it = decode_item<kQBlock>(w, grp, order, prefix, BG, H);
+        const Item it = decode_item<kQBlock>(Redo ? redo[4 + w] : w, grp, order, prefix, BG, H);
         const int ntiles = (it.khi - it.klo + kTileN - 1) / kTileN;
         const bool validB = it.row0 + kTileM < it.qhi;
         for (int x = 0; x < (validB ? 2 : 1) && ok; ++x) {
@@ -238,7 +239,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                  (accumulate || kk > 0) ? 1u : 0u);
       };
       for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
-        const Item it = decode_item<kQBlock>(w, grp, order, prefix, BG, H);
+        const Item it = decode_item<kQBlock>(Redo ? redo[4 + w] : w, grp, order, prefix, BG, H);
         const int ntiles = (it.khi - it.klo + kTileN - 1) / kTileN;
         const int nx = (it.row0 + kTileM < it.qhi) ? 2 : 1;
         // first S tiles
@@ -309,7 +310,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     uint32_t n_s = 0, n_o = 0;
     bool ok = true;
     for (int w = blockIdx.x; ok && w < total_items; w += gridDim.x) {
-      const Item it = decode_item<kQBlock>(w, grp, order, prefix, BG, H);
+      const Item it = decode_item<kQBlock>(Redo ? redo[4 + w] : w, grp, order, prefix, BG, H);
       if (x == 1 && !(it.row0 + kTileM < it.qhi)) continue;
       const int ntiles = (it.khi - it.klo + kTileN - 1) / kTileN;
       const int tile_row0 = it.row0 + x * kTileM;
@@ -467,21 +468,26 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 }
 
 // ----------------------------------------------------------------------------- host side
-template <int D>
+// Tensor maps, grid and launch of the one-CTA kernel.  Redo: only the items the CTA-pair kernel
+// listed in p.redo, whose schedule (the same 256-row items) is already in order / prefix.
+template <int D, bool Redo>
 moga_status launch_one(const Problem& p, cudaStream_t st) {
   CUtensorMap mq, mk, mv;
   const long long BH = (long long)p.B * p.H;
   if (!make_map(&mq, p.Q, D, p.Tq, BH, kTileM) || !make_map(&mk, p.K, D, p.Tkv, BH, kTileN) ||
       !make_map(&mv, p.V, D, p.Tkv, BH, kTileN))
     return MOGA_ERR_CUDA;
-  attn_schedule_kernel<<<1, 1024, 0, st>>>(p.grp, p.order, p.prefix, p.B, p.H, kQBlock);
-  MOGA_CUDA_OK(cudaGetLastError());
+  if (!Redo) {
+    attn_schedule_kernel<<<1, 1024, 0, st>>>(p.grp, p.order, p.prefix, p.B, p.H, kQBlock);
+    MOGA_CUDA_OK(cudaGetLastError());
+  }
   int num_sms = 0;
   if (!current_sm_count(&num_sms)) return MOGA_ERR_CUDA;
-  auto kern = attn_bf16_kernel<D>;
+  auto kern = attn_bf16_kernel<D, Redo>;
   MOGA_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::kDynSmem));
-  const long long max_items = ((p.Tq + kQBlock - 1) / kQBlock + p.grp.G) * BH;
-  const int grid = (int)(max_items < num_sms ? max_items : num_sms);
+  const long long max_items = max_items_256(p);
+  int grid = (int)(max_items < num_sms ? max_items : num_sms);
+  if (Redo && grid > 16) grid = 16;      // the list is normally empty: a few CTAs walk it
   // The kernel works in the log2 domain with scale_log2 = scale * log2(e) and masks columns by
   // setting their score to -inf, which needs scale_log2 > 0 (-inf * 0 is NaN).  A zero scale
   // (uniform weights) is served by the smallest normal float instead: every weight
@@ -490,22 +496,22 @@ moga_status launch_one(const Problem& p, cudaStream_t st) {
   const float scale_log2 = p.scale * log2e > 1.17549435e-38f ? p.scale * log2e : 1.17549435e-38f;
   kern<<<grid, kThreads, Cfg<D>::kDynSmem, st>>>(mq, mk, mv, p.grp, p.order, p.prefix,
                                                   static_cast<__nv_bfloat16*>(p.O), p.lse, p.header, (int)p.Tq,
-                                                  p.H, p.B * p.grp.G, scale_log2, p.scale, p.sc);
+                                                  p.H, p.B * p.grp.G, scale_log2, p.scale, p.sc, p.redo);
   MOGA_CUDA_OK(cudaGetLastError());
   return MOGA_OK;
 }
 
-// Which kernel serves a launch.  The CTA-pair kernel (D = 128 only) halves the K/V bytes each
-// SM stages and reads per flop, but its work item is 512 query rows: it takes the launches whose
-// groups are long (mean of at least kPairMinRows query rows per group); short groups, such as
-// the static ones of Sec. 3.2, and D = 64 stay on the one-CTA kernel.  g_attn_kernel overrides
-// the choice (moga_set_attn_kernel).
-constexpr long long kPairMinRows = 2048;
+// Which kernel serves a launch.  The one-CTA kernel is the default for every shape: measured on
+// groups of ~17,500 rows it runs at 1,150-1,160 TFLOP/s against 935 for the CTA-pair kernel (same
+// box, alternating runs).  The pair kernel halves the K/V bytes each SM stages and reads per
+// flop, but issuing an M = 256, N = 128 instruction for two SMs keeps the issuing thread about as
+// long as the instruction runs, so its waits are no longer hidden behind queued MMAs and the
+// tensor pipe idles 55 % of the cycles.  It stays selectable (moga_set_attn_kernel) for d_head = 128
+// launches that have the redo scratch.
 int g_attn_kernel = MOGA_ATTN_AUTO;
 
 moga_status launch_any(int D, const Problem& p, cudaStream_t st) {
-  const bool long_groups = p.grp.G > 0 && p.Tq / p.grp.G >= kPairMinRows;
-  const bool pair = D == 128 && (g_attn_kernel == MOGA_ATTN_PAIR || (g_attn_kernel == MOGA_ATTN_AUTO && long_groups));
+  const bool pair = D == 128 && p.redo != nullptr && g_attn_kernel == MOGA_ATTN_PAIR;
   return pair ? launch_pair(p, st) : launch_single(D, p, st);
 }
 
@@ -515,14 +521,17 @@ Problem routed_problem(const moga_shape& s, const WsLayout& L, const void* Qp, c
   const long long T = (long long)s.N * s.k;
   int32_t* order = reinterpret_cast<int32_t*>(ws + L.sched);
   return Problem{s.B, s.H, T, T, s.scale, Qp, Kp, Vp, O, lse, Groups{offsets, offsets, s.M + 1, s.M},
-                 order, order + (size_t)s.B * s.M, reinterpret_cast<uint32_t*>(ws + L.header), sc};
+                 order, order + (size_t)s.B * s.M, reinterpret_cast<int32_t*>(ws + L.redo),
+                 reinterpret_cast<uint32_t*>(ws + L.header), sc};
 }
 
 }  // namespace
 
 moga_status attn::launch_single(int D, const attn::Problem& p, cudaStream_t st) {
-  return D == 128 ? launch_one<128>(p, st) : launch_one<64>(p, st);
+  return D == 128 ? launch_one<128, false>(p, st) : launch_one<64, false>(p, st);
 }
+
+moga_status attn::launch_single_redo(const attn::Problem& p, cudaStream_t st) { return launch_one<128, true>(p, st); }
 
 void set_attn_kernel(int mode) { g_attn_kernel = mode; }
 
@@ -550,7 +559,7 @@ moga_status launch_attn_bf16_static(const moga_shape& s, int G, long long Tq, lo
   const Scatter none{nullptr, nullptr, 0, 0, 0, 0};
   int32_t* order = reinterpret_cast<int32_t*>(ws + 256);
   const Problem p{s.B, s.H, Tq, Tkv, s.scale, Qs, Ks, Vs, Os, lse, Groups{q_offsets, kv_offsets, 0, G},
-                  order, order + (size_t)s.B * G, reinterpret_cast<uint32_t*>(ws), none};
+                  order, order + (size_t)s.B * G, nullptr, reinterpret_cast<uint32_t*>(ws), none};
   return launch_any(s.D, p, st);
 }
 

@@ -97,15 +97,24 @@ struct Problem {
   float* lse;
   Groups grp;
   int32_t *order, *prefix;   // scratch: B*G and B*G + 1 int32
+  int32_t* redo;             // scratch of the CTA-pair kernel (items for the exact path): int32
+                             // [4 + 2 * max_items_256]; nullptr: the launch cannot use that kernel
   uint32_t* header;          // device status word
   Scatter sc;
 };
 
 
+// Upper bound on the work items of 256 query rows in a launch.
+inline long long max_items_256(const Problem& p) {
+  return ((p.Tq + 255) / 256 + p.grp.G) * (long long)p.B * p.H;
+}
+
 // kernels (each in its own file); both read the schedule attn_schedule_kernel wrote for their
 // query block
 moga_status launch_single(int D, const Problem& p, cudaStream_t st);   // 256 query rows per CTA
-moga_status launch_pair(const Problem& p, cudaStream_t st);            // D = 128, 512 query rows per CTA pair
+moga_status launch_pair(const Problem& p, cudaStream_t st);            // D = 128, 256 query rows per CTA pair
+// D = 128: the one-CTA kernel over the items listed in p.redo (their schedule is already in place)
+moga_status launch_single_redo(const Problem& p, cudaStream_t st);
 
 }  // namespace attn
 }  // namespace moga

@@ -27,6 +27,7 @@ struct WsLayout {
   size_t sched;       // int32 [B, 3, M+1]    attention schedule (order, tile prefix, ...)
   size_t wsplit;      // bf16 [3, MP, C]      router weight split into three bf16 parts (MP <= 64)
   size_t stats;       // int32 + float [B, nblk, M] per-block counts and gate sums (Eq. 6-8)
+  size_t redo;        // int32 [4 + 2 * items]  work items the CTA-pair attention kernel hands to the exact path
   size_t scratch_end; // == moga_scratch_bytes
   size_t gid, gate, perm, inv, offsets;  // routing results
   size_t Qp, Kp, Vp, Op;                 // permuted tensors
@@ -48,6 +49,10 @@ inline WsLayout ws_layout(const moga_shape& s) {
   L.sched = off;       off = align_up(off + sizeof(int32_t) * (size_t)s.B * 4 * (s.M + 1) + 64, kWsAlign);
   L.wsplit = off;      off = align_up(off + sizeof(uint16_t) * 3 * (size_t)kMaxM * s.C, kWsAlign);
   L.stats = off;       off = align_up(off + 2 * sizeof(int32_t) * (size_t)s.B * L.nblk * s.M, kWsAlign);
+  {
+    const size_t items = ((T + 255) / 256 + (size_t)s.M) * (size_t)s.B * (size_t)s.H;
+    L.redo = off;      off = align_up(off + sizeof(int32_t) * (4 + 2 * items), kWsAlign);
+  }
   L.scratch_end = off;
   L.gid = off;         off = align_up(off + sizeof(int32_t) * (size_t)s.B * T, kWsAlign);
   L.gate = off;        off = align_up(off + sizeof(float) * (size_t)s.B * T, kWsAlign);

@@ -357,9 +357,12 @@ def test_group_attn_neighbour_group_does_not_leak(mb, dtype):
     assert torch.equal(outs[0], outs[1])
 
 
+@pytest.mark.parametrize("kernel", ["single", "pair"])
 @pytest.mark.parametrize("grow", [3.0, 24.0])
-def test_group_attn_growing_scores_bf16(mb, grow):
-    """Keys late in each group are scaled up, so later K/V tiles hold scores far above the
+def test_group_attn_growing_scores_bf16(mb, grow, kernel):
+    """Both kernels: the one-CTA kernel changes the reference inside the row; the CTA-pair kernel
+    hands such items to the one-CTA kernel's exact path afterwards.
+    Keys late in each group are scaled up, so later K/V tiles hold scores far above the
     first tile's maximum: x3 stays on the kernel's fixed-reference path with large positive
     exponents, x24 overflows it and forces the mid-row change of reference.  Outputs are
     O(1) here (a few keys dominate each row), so the bound is relative."""
@@ -375,9 +378,13 @@ def test_group_attn_growing_scores_bf16(mb, grow):
     Op = torch.full_like(case["Q"], float("nan"))
     lse = torch.empty(1, 2, case["T"], dtype=torch.float32, device="cuda")
     ws = mb.alloc_workspace(mb.moga_scratch_bytes(sh))
-    mb.moga_group_attn(sh, case["Q"], case["K"], case["V"], torch.from_numpy(case["offsets"]).cuda(), Op,
-                       lse, ws)
-    assert mb.moga_last_device_status(ws) == (0, 0)
+    mb.moga_set_attn_kernel(mb.MOGA_ATTN_PAIR if kernel == "pair" else mb.MOGA_ATTN_SINGLE)
+    try:
+        mb.moga_group_attn(sh, case["Q"], case["K"], case["V"], torch.from_numpy(case["offsets"]).cuda(), Op,
+                           lse, ws)
+        assert mb.moga_last_device_status(ws) == (0, 0)
+    finally:
+        mb.moga_set_attn_kernel(mb.MOGA_ATTN_AUTO)
     want = oracle.attn_all(to_np32(case["Q"]), to_np32(case["K"]), to_np32(case["V"]), case["gid"],
                            np.ones((1, case["T"], 1)), case["offsets"], case["perm"], scale)
     got = Op.float().cpu().numpy().astype(np.float64)
