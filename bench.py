@@ -233,10 +233,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--sharding", default="layers", choices=["layers", "heads"],
-                    help="with --gpus N > 1: 'layers' gives every rank its own layer (weak scaling, no collective); "
-                         "'heads' splits ONE layer: tokens of X for routing, heads of Q/K/V for attention, with the "
-                         "all-gather of the routing results as the only exchange (strong scaling)")
+    ap.add_argument("--sharding", default="auto", choices=["auto", "layers", "heads"],
+                    help="with N > 1 ranks: 'heads' splits ONE layer: tokens of X for routing, heads of Q/K/V for "
+                         "attention, with one all-gather of the routing results as the only exchange (strong "
+                         "scaling; the default for N > 1); 'layers' gives every rank its own layer (weak scaling, no "
+                         "collective; the default for N = 1)")
     ap.add_argument("--stage", default="all", choices=["all", "route", "visual"],
                     help="'route' times moga_route alone on the config's X (a small resident set, for profiling); "
                          "'visual' times the whole visual-attention block: routed branch, the two static-group "
@@ -259,6 +260,8 @@ def main():
     from paper_2510_18692_b200 import binding as mb   # raises if the CUDA library is missing
 
     cfg = cfg.with_(seed=cfg.seed + 100 * rank)       # every rank works on its own layer
+    if args.sharding == "auto":
+        args.sharding = "heads" if world > 1 else "layers"
     if args.sharding == "heads":
         return run_head_sharded(mb, CONFIGS[args.config], dev, args, rank, world)
     if args.stage == "route":
@@ -436,16 +439,17 @@ def run_route_only(mb, cfg, dev, args):
 
 def run_head_sharded(mb, cfg, dev, args, rank, world):
     """One layer split over the ranks (strong scaling): see paper_2510_18692_b200/sharded.py."""
-    from paper_2510_18692_b200.sharded import forward_head_sharded, shard_bounds
+    from paper_2510_18692_b200.sharded import ShardPlan, shard_bounds
     lo, hi = shard_bounds(cfg.N, world, rank)
     h_lo, h_hi = shard_bounds(cfg.H, world, rank)
     inp = make_inputs(cfg, device=dev, heads=list(range(h_lo, h_hi)))      # every rank draws the same layer
     X_local = inp["X"][:, lo:hi].contiguous()
     del inp["X"]
     O = torch.empty_like(inp["Q"])
+    plan = ShardPlan(mb, cfg, dev)          # workspaces, routing and exchange buffers: allocated once
 
     def step():
-        return forward_head_sharded(mb, cfg, X_local, inp["Wr"], inp["bias"], inp["Q"], inp["K"], inp["V"], O)
+        return plan.forward(X_local, inp["Wr"], inp["bias"], inp["Q"], inp["K"], inp["V"], O)
 
     for _ in range(args.warmup):
         _, _, offsets = step()
@@ -472,7 +476,8 @@ def run_head_sharded(mb, cfg, dev, args, rank, world):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "strong", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
             "config": dict(config_dict(cfg), sharding="tokens for routing, heads for attention; one all-gather of (gid, gate)"),
-            "gpu_launches": (kernels_per_forward(cfg) + (1 if cfg.k == 1 and cfg.dtype == "bf16" else 0)) * args.steps,
+            "gpu_launches": kernels_per_forward(cfg) * args.steps,
+            "ms_per_layer_head_batch": ms * world / (cfg.B * cfg.H),
             "clocks": clk}))
     return 0
 

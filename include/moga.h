@@ -277,6 +277,19 @@ moga_status moga_forward(const moga_shape* s, const void* X, const float* Wr, co
                          size_t ws_bytes, void* stream);
 
 /*
+ * The same forward from a routing that is already known (Alg. 1 lines 2-4 and the gate of
+ * Eq. 5, without the router of Eq. 2-4): gid and gate [B, N, k] as moga_route writes them.
+ * This is the call of a rank that holds only some heads of Q, K, V (shape.H = its heads) and
+ * received the routing of the whole sequence from the ranks that hold the token features
+ * (Sec. 3.2, last paragraph: routing is computed per token before the model's sequence-to-head
+ * exchange and its results are gathered).  Same kernels, workspace (moga_workspace_bytes) and
+ * results as moga_forward given the same routing.  perm_out / offsets_out may be NULL.
+ */
+moga_status moga_forward_routed(const moga_shape* s, const int32_t* gid, const float* gate, const void* Q,
+                                const void* K, const void* V, void* O, int32_t* perm_out, int32_t* offsets_out,
+                                void* ws, size_t ws_bytes, void* stream);
+
+/*
  * The whole forward from HOST buffers (the call for a caller whose activations live in host
  * memory).  X, Wr, bias, Q, K, V, O, gid_out, gate_out are HOST pointers (page-locked memory
  * is needed for the copies to overlap; pageable memory works but serialises); Q, K, V, O are

@@ -21,7 +21,7 @@ EXPORTS = ("moga_workspace_bytes", "moga_scratch_bytes", "moga_status_string", "
            "moga_permute", "moga_group_attn", "moga_unpermute", "moga_forward",
            "moga_last_device_status", "moga_sort_static", "moga_balance_stats", "moga_stga_build", "moga_gather_rows",
            "moga_static_group_attn", "moga_mean3", "moga_forward_host_bytes", "moga_forward_host",
-           "moga_visual_workspace_bytes", "moga_visual_forward", "moga_selftest_wait_timeout", "moga_set_attn_kernel")
+           "moga_visual_workspace_bytes", "moga_visual_forward", "moga_selftest_wait_timeout", "moga_set_attn_kernel", "moga_forward_routed")
 
 MOGA_F32, MOGA_BF16 = 0, 1
 MOGA_ROUTE_AUTO, MOGA_ROUTE_ALU = 0, 1
@@ -185,6 +185,12 @@ def moga_forward(shape, X, Wr, bias, Q, K, V, O, ws, gid_out=None, gate_out=None
            "moga_forward")
 
 
+def moga_forward_routed(shape, gid, gate, Q, K, V, O, ws, perm_out=None, offsets_out=None):
+    _check(lib.moga_forward_routed(ctypes.byref(shape), _ptr(gid), _ptr(gate), _ptr(Q), _ptr(K), _ptr(V), _ptr(O),
+                                   _ptr(perm_out), _ptr(offsets_out), _ptr(ws), ctypes.c_size_t(ws.numel()),
+                                   _stream()), "moga_forward_routed")
+
+
 def moga_forward_host_bytes(shape, heads_per_chunk) -> int:
     return int(lib.moga_forward_host_bytes(ctypes.byref(shape), ctypes.c_int32(heads_per_chunk)))
 
@@ -218,7 +224,7 @@ def moga_visual_forward(shape, X, Wr, bias, Q, K, V, O, static_lists, ws):
 
 def moga_selftest_wait_timeout(ws, limit_ns):
     _check(lib.moga_selftest_wait_timeout(_ptr(ws), ctypes.c_size_t(ws.numel()), ctypes.c_uint64(limit_ns),
-                                          _stream()), "moga_selftest_wait_timeout", "moga_set_attn_kernel")
+                                          _stream()), "moga_selftest_wait_timeout")
 
 
 MOGA_ATTN_AUTO, MOGA_ATTN_SINGLE, MOGA_ATTN_PAIR = 0, 1, 2

@@ -93,7 +93,7 @@ struct Cfg {
 };
 
 // Redo: the work items are those listed in redo[4 ...] (redo[0] of them) instead of all items.
-template <int D, bool Redo>
+template <int D, bool Redo, int Epi>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                  const __grid_constant__ CUtensorMap mapV, const Groups grp,
@@ -394,6 +394,22 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       }
       if (!ok) break;
       // ---- epilogue: O / l -> bf16 -> per-warp staging -> global
+      // mean of three branches: the rows of the other two branches this lane will need (4 rows x
+      // 4 column chunks x 16 bytes of each) are requested now, so they arrive while the item's
+      // last P V runs; the softmax registers are free at this point
+      uint4 pre_a[D / 32][4], pre_b[D / 32][4];
+      if (Epi == kEpiMean3) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int grow = tile_row0 + q * 32 + i * 8 + (lane >> 2);
+          const long long at = ((long long)it.bh * T + (grow < it.qhi ? grow : it.qhi - 1)) * D + (lane & 3) * 8;
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            pre_a[c][i] = __ldg(reinterpret_cast<const uint4*>(sc.mean_a + at + c * 32));
+            pre_b[c][i] = __ldg(reinterpret_cast<const uint4*>(sc.mean_b + at + c * 32));
+          }
+        }
+      }
       ok = __all_sync(0xffffffffu, wait(O_FULL + x, n_o & 1u, 11));
       if (!ok) break;
       ++n_o;
@@ -401,7 +417,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       float inv_l = 1.f / l;
       const bool live = tile_row0 + r < it.qhi;
       const int bb = it.bh / H, hh = it.bh % H;
-      if (sc.perm != nullptr && live) inv_l *= sc.gate[(size_t)bb * sc.N + sc.perm[(size_t)bb * T + tile_row0 + r]];
+      if (Epi == kEpiDefault && sc.perm != nullptr && live)
+        inv_l *= sc.gate[(size_t)bb * sc.N + sc.perm[(size_t)bb * T + tile_row0 + r]];
       // Each warp stages 32 rows x 32 columns (2 KB) at a time in its own buffer and writes them
       // out itself: lane L stores piece L % 4 of rows i * 8 + L / 4, i = 0..3 (64-byte row segments).
       unsigned char* wst = smem + C::kSmemStage + (x * 4 + q) * 2048;
@@ -411,7 +428,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       for (int i = 0; i < 4; ++i) {
         const int grow = tile_row0 + q * 32 + i * 8 + (lane >> 2);
         orow_live[i] = grow < it.qhi;
-        if (sc.perm != nullptr) {
+        if (Epi == kEpiList) {
+          const int tok = orow_live[i] ? sc.perm[grow] : 0;
+          obase[i] = Op + bb * sc.sb + hh * sc.sh + (long long)tok * sc.sn;
+        } else if (Epi == kEpiDefault && sc.perm != nullptr) {
           const int tok = orow_live[i] ? sc.perm[(size_t)bb * T + grow] : 0;
           obase[i] = Op + bb * sc.sb + hh * sc.sh + (long long)tok * sc.sn;
         } else {
@@ -443,7 +463,22 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int row = i * 8 + (lane >> 2), piece = lane & 3;
-          const uint4 val = *reinterpret_cast<const uint4*>(wst + row * 64 + ((piece ^ ((row >> 1) & 3)) * 16));
+          uint4 val = *reinterpret_cast<const uint4*>(wst + row * 64 + ((piece ^ ((row >> 1) & 3)) * 16));
+          if (Epi == kEpiMean3) {
+            // the other two branches' rows live at the same offset of their own tensors
+            const uint4 a = pre_a[c][i], b = pre_b[c][i];
+            const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+            uint32_t* vw = reinterpret_cast<uint32_t*>(&val);
+            const float third = 1.f / 3.f;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float lo = (__uint_as_float(aw[e] << 16) + __uint_as_float(bw[e] << 16)) + __uint_as_float(vw[e] << 16);
+              const float hi = (__uint_as_float(aw[e] & 0xffff0000u) + __uint_as_float(bw[e] & 0xffff0000u)) +
+                               __uint_as_float(vw[e] & 0xffff0000u);
+              __nv_bfloat162 t = __floats2bfloat162_rn(lo * third, hi * third);
+              vw[e] = *reinterpret_cast<uint32_t*>(&t);
+            }
+          }
           if (orow_live[i]) *reinterpret_cast<uint4*>(obase[i] + c * 32 + piece * 8) = val;
         }
         __syncwarp();
@@ -470,7 +505,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 // ----------------------------------------------------------------------------- host side
 // Tensor maps, grid and launch of the one-CTA kernel.  Redo: only the items the CTA-pair kernel
 // listed in p.redo, whose schedule (the same 256-row items) is already in order / prefix.
-template <int D, bool Redo>
+template <int D, bool Redo, int Epi>
 moga_status launch_one(const Problem& p, cudaStream_t st) {
   CUtensorMap mq, mk, mv;
   const long long BH = (long long)p.B * p.H;
@@ -483,7 +518,7 @@ moga_status launch_one(const Problem& p, cudaStream_t st) {
   }
   int num_sms = 0;
   if (!current_sm_count(&num_sms)) return MOGA_ERR_CUDA;
-  auto kern = attn_bf16_kernel<D, Redo>;
+  auto kern = attn_bf16_kernel<D, Redo, Epi>;
   MOGA_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::kDynSmem));
   const long long max_items = max_items_256(p);
   int grid = (int)(max_items < num_sms ? max_items : num_sms);
@@ -511,7 +546,7 @@ moga_status launch_one(const Problem& p, cudaStream_t st) {
 int g_attn_kernel = MOGA_ATTN_AUTO;
 
 moga_status launch_any(int D, const Problem& p, cudaStream_t st) {
-  const bool pair = D == 128 && p.redo != nullptr && g_attn_kernel == MOGA_ATTN_PAIR;
+  const bool pair = D == 128 && p.redo != nullptr && p.epi == kEpiDefault && g_attn_kernel == MOGA_ATTN_PAIR;
   return pair ? launch_pair(p, st) : launch_single(D, p, st);
 }
 
@@ -522,16 +557,18 @@ Problem routed_problem(const moga_shape& s, const WsLayout& L, const void* Qp, c
   int32_t* order = reinterpret_cast<int32_t*>(ws + L.sched);
   return Problem{s.B, s.H, T, T, s.scale, Qp, Kp, Vp, O, lse, Groups{offsets, offsets, s.M + 1, s.M},
                  order, order + (size_t)s.B * s.M, reinterpret_cast<int32_t*>(ws + L.redo),
-                 reinterpret_cast<uint32_t*>(ws + L.header), sc};
+                 reinterpret_cast<uint32_t*>(ws + L.header), sc, kEpiDefault};
 }
 
 }  // namespace
 
 moga_status attn::launch_single(int D, const attn::Problem& p, cudaStream_t st) {
-  return D == 128 ? launch_one<128, false>(p, st) : launch_one<64, false>(p, st);
+  if (p.epi == kEpiList) return D == 128 ? launch_one<128, false, kEpiList>(p, st) : MOGA_ERR_UNSUPPORTED;
+  if (p.epi == kEpiMean3) return D == 128 ? launch_one<128, false, kEpiMean3>(p, st) : MOGA_ERR_UNSUPPORTED;
+  return D == 128 ? launch_one<128, false, kEpiDefault>(p, st) : launch_one<64, false, kEpiDefault>(p, st);
 }
 
-moga_status attn::launch_single_redo(const attn::Problem& p, cudaStream_t st) { return launch_one<128, true>(p, st); }
+moga_status attn::launch_single_redo(const attn::Problem& p, cudaStream_t st) { return launch_one<128, true, kEpiDefault>(p, st); }
 
 void set_attn_kernel(int mode) { g_attn_kernel = mode; }
 
@@ -539,7 +576,7 @@ moga_status launch_attn_bf16(const moga_shape& s, const WsLayout& L, const void*
                              const void* Vp, const int32_t* offsets, void* Op, float* lse, char* ws,
                              cudaStream_t st) {
   if ((long long)s.N * s.k == 0) return MOGA_OK;
-  const Scatter none{nullptr, nullptr, 0, 0, 0, 0};
+  const Scatter none{nullptr, nullptr, 0, 0, 0, 0, nullptr, nullptr};
   return launch_any(s.D, routed_problem(s, L, Qp, Kp, Vp, offsets, Op, lse, ws, none), st);
 }
 
@@ -548,18 +585,32 @@ moga_status launch_attn_bf16_scatter(const moga_shape& s, const WsLayout& L, con
                                      const float* gate, void* O, char* ws, cudaStream_t st) {
   if ((long long)s.N * s.k == 0) return MOGA_OK;
   const Strides q = qkv_strides(s);
-  const Scatter sc{perm, gate, q.b, q.h, q.n, s.N};
+  const Scatter sc{perm, gate, q.b, q.h, q.n, s.N, nullptr, nullptr};
   return launch_any(s.D, routed_problem(s, L, Qp, Kp, Vp, offsets, O, nullptr, ws, sc), st);
 }
 
 moga_status launch_attn_bf16_static(const moga_shape& s, int G, long long Tq, long long Tkv, const void* Qs,
                                     const void* Ks, const void* Vs, const int32_t* q_offsets,
-                                    const int32_t* kv_offsets, void* Os, float* lse, char* ws, cudaStream_t st) {
+                                    const int32_t* kv_offsets, void* Os, float* lse, uint32_t* header, char* sched,
+                                    const StaticEpilogue& epi, cudaStream_t st) {
   if (Tq == 0 || G == 0) return MOGA_OK;
-  const Scatter none{nullptr, nullptr, 0, 0, 0, 0};
-  int32_t* order = reinterpret_cast<int32_t*>(ws + 256);
+  Scatter sc{nullptr, nullptr, 0, 0, 0, 0, nullptr, nullptr};
+  int mode = attn::kEpiDefault;
+  if (epi.token_list != nullptr) {          // rows go to token order: Os is [B, H, N, D]
+    mode = attn::kEpiList;
+    sc.perm = epi.token_list;
+    sc.sb = (long long)s.H * s.N * s.D;
+    sc.sh = (long long)s.N * s.D;
+    sc.sn = s.D;
+    sc.N = s.N;
+  } else if (epi.mean_a != nullptr) {       // mean with two token-order tensors: rows stay in place
+    mode = attn::kEpiMean3;
+    sc.mean_a = static_cast<const __nv_bfloat16*>(epi.mean_a);
+    sc.mean_b = static_cast<const __nv_bfloat16*>(epi.mean_b);
+  }
+  int32_t* order = reinterpret_cast<int32_t*>(sched);
   const Problem p{s.B, s.H, Tq, Tkv, s.scale, Qs, Ks, Vs, Os, lse, Groups{q_offsets, kv_offsets, 0, G},
-                  order, order + (size_t)s.B * G, nullptr, reinterpret_cast<uint32_t*>(ws), none};
+                  order, order + (size_t)s.B * G, nullptr, header, sc, mode};
   return launch_any(s.D, p, st);
 }
 

@@ -63,15 +63,25 @@ __device__ __forceinline__ Item decode_item(int w, const Groups& grp, const int3
   return it;
 }
 
-// Output placement.  perm == nullptr: rows stay in sorted order, Op is [B*H, T, D].
-// Otherwise (top-1 routing) the epilogue is the gated inverse permutation of Eq. 5: sorted
-// row p of batch item b goes to token perm[b, p] of O (element strides sb, sh, sn),
-// multiplied by gate[b, token] in fp32 before the one rounding to bf16.
+// Output placement (the kernels' epilogue).
+//   kEpiDefault   perm == nullptr: rows stay in sorted order, Op is [B*H, T, D].  Otherwise
+//                 (top-1 routing) the gated inverse permutation of Eq. 5: sorted row p of batch
+//                 item b goes to token perm[b, p] of O (element strides sb, sh, sn), multiplied
+//                 by gate[b, token] in fp32 before the one rounding to bf16.
+//   kEpiList      static groups: row p goes to token perm[p] (one list for all batch items), no
+//                 gate.
+//   kEpiMean3     last branch of the visual attention block (Sec. 3.2): rows stay in place
+//                 (contiguous [B, H, N, D]); the stored value is the mean of this branch's row,
+//                 rounded to bf16 as if it had been stored, and the rows of mean_a and mean_b at
+//                 the same place: (a + b + c) / 3 in fp32, one rounding.
+constexpr int kEpiDefault = 0, kEpiList = 1, kEpiMean3 = 2;
 struct Scatter {
   const int32_t* perm;
   const float* gate;
   long long sb, sh, sn;
   int N;
+  const __nv_bfloat16* mean_a;
+  const __nv_bfloat16* mean_b;
 };
 
 // [B*H, T, D] bf16, box 64 columns x box_rows rows x 1, 128-byte swizzle, out-of-range rows read as zero.
@@ -101,6 +111,7 @@ struct Problem {
                              // [4 + 2 * max_items_256]; nullptr: the launch cannot use that kernel
   uint32_t* header;          // device status word
   Scatter sc;
+  int epi;                   // kEpiDefault / kEpiList / kEpiMean3 (the latter two: one-CTA kernel, D = 128)
 };
 
 

@@ -207,7 +207,8 @@ moga_status moga_static_group_attn(const moga_shape* s, int32_t G, int32_t Tq, i
     return launch_attn_f32_groups(s->B, s->H, s->D, s->scale, G, Tq, Tkv, static_cast<const float*>(Qs),
                                   static_cast<const float*>(Ks), static_cast<const float*>(Vs), q_offsets,
                                   kv_offsets, 0, static_cast<float*>(Os), lse, cs);
-  return launch_attn_bf16_static(*s, G, Tq, Tkv, Qs, Ks, Vs, q_offsets, kv_offsets, Os, lse, w, cs);
+  return launch_attn_bf16_static(*s, G, Tq, Tkv, Qs, Ks, Vs, q_offsets, kv_offsets, Os, lse,
+                                 reinterpret_cast<uint32_t*>(w), w + 256, StaticEpilogue{nullptr, nullptr, nullptr}, cs);
 }
 
 moga_status moga_mean3(const moga_shape* s, const void* A, const void* Bs, const int32_t* inv_b,
@@ -226,6 +227,43 @@ moga_status moga_unpermute(const moga_shape* s, const void* Op, const int32_t* i
   if (!PTR_OK(Op) || !PTR_OK(inv) || !PTR_OK(gate) || !PTR_OK(O)) return MOGA_ERR_INVALID_ARG;
   return launch_unpermute(*s, Op, inv, gate, O, static_cast<cudaStream_t>(stream));
 }
+
+}  // extern "C"
+
+namespace {
+// Alg. 1 lines 2-4 and the gate of Eq. 5 from a given routing: sort, gather, group attention,
+// gated inverse permutation, with the intermediates in the forward workspace.
+moga_status forward_after_route(const moga_shape* s, const WsLayout& L, const int32_t* gid, const float* gate,
+                                const void* Q, const void* K, const void* V, void* O, int32_t* perm_out,
+                                int32_t* offsets_out, char* w, cudaStream_t cs) {
+  moga_status st;
+  int32_t* perm = reinterpret_cast<int32_t*>(w + L.perm);
+  int32_t* inv = reinterpret_cast<int32_t*>(w + L.inv);
+  int32_t* offsets = reinterpret_cast<int32_t*>(w + L.offsets);
+  void* Qp = w + L.Qp;
+  void* Kp = w + L.Kp;
+  void* Vp = w + L.Vp;
+  void* Op = w + L.Op;
+  if ((st = launch_sort(*s, L, gid, perm, inv, offsets, w, cs)) != MOGA_OK) return st;
+  if ((st = launch_gather(*s, perm, Q, K, V, Qp, Kp, Vp, cs)) != MOGA_OK) return st;
+  if (s->dtype == MOGA_F32)
+    st = launch_attn_f32(*s, static_cast<const float*>(Qp), static_cast<const float*>(Kp),
+                         static_cast<const float*>(Vp), offsets, static_cast<float*>(Op), nullptr, cs);
+  else if (s->k == 1)   // one assignment per token: the attention epilogue is the gated scatter
+    st = launch_attn_bf16_scatter(*s, L, Qp, Kp, Vp, offsets, perm, gate, O, w, cs);
+  else
+    st = launch_attn_bf16(*s, L, Qp, Kp, Vp, offsets, Op, nullptr, w, cs);
+  if (st != MOGA_OK) return st;
+  if (s->dtype == MOGA_F32 || s->k > 1)
+    if ((st = launch_unpermute(*s, Op, inv, gate, O, cs)) != MOGA_OK) return st;
+  const size_t T = (size_t)s->N * s->k;
+  if (perm_out) MOGA_CUDA_OK(cudaMemcpyAsync(perm_out, perm, sizeof(int32_t) * s->B * T, cudaMemcpyDeviceToDevice, cs));
+  if (offsets_out) MOGA_CUDA_OK(cudaMemcpyAsync(offsets_out, offsets, sizeof(int32_t) * s->B * (s->M + 1), cudaMemcpyDeviceToDevice, cs));
+  return MOGA_OK;
+}
+}  // namespace
+
+extern "C" {
 
 moga_status moga_forward(const moga_shape* s, const void* X, const float* Wr, const float* bias,
                          const void* Q, const void* K, const void* V, void* O, int32_t* gid_out,
@@ -247,37 +285,40 @@ moga_status moga_forward(const moga_shape* s, const void* X, const float* Wr, co
   char* w = static_cast<char*>(ws);
   int32_t* gid = reinterpret_cast<int32_t*>(w + L.gid);
   float* gate = reinterpret_cast<float*>(w + L.gate);
-  int32_t* perm = reinterpret_cast<int32_t*>(w + L.perm);
-  int32_t* inv = reinterpret_cast<int32_t*>(w + L.inv);
-  int32_t* offsets = reinterpret_cast<int32_t*>(w + L.offsets);
-  void* Qp = w + L.Qp;
-  void* Kp = w + L.Kp;
-  void* Vp = w + L.Vp;
-  void* Op = w + L.Op;
   if ((st = clear_header(w, L, cs)) != MOGA_OK) return st;
   st = route_on_tensor_cores(*s, L, ws, ws_bytes)
            ? launch_route_mma(*s, L, X, Wr, bias, gid, gate, nullptr, w, cs)
            : launch_route(*s, X, Wr, bias, gid, gate, nullptr, cs);
   if (st != MOGA_OK) return st;
-  if ((st = launch_sort(*s, L, gid, perm, inv, offsets, w, cs)) != MOGA_OK) return st;
-  if ((st = launch_gather(*s, perm, Q, K, V, Qp, Kp, Vp, cs)) != MOGA_OK) return st;
-  if (s->dtype == MOGA_F32)
-    st = launch_attn_f32(*s, static_cast<const float*>(Qp), static_cast<const float*>(Kp),
-                         static_cast<const float*>(Vp), offsets, static_cast<float*>(Op), nullptr, cs);
-  else if (s->k == 1)   // one assignment per token: the attention epilogue is the gated scatter
-    st = launch_attn_bf16_scatter(*s, L, Qp, Kp, Vp, offsets, perm, gate, O, w, cs);
-  else
-    st = launch_attn_bf16(*s, L, Qp, Kp, Vp, offsets, Op, nullptr, w, cs);
-  if (st != MOGA_OK) return st;
-  if (s->dtype == MOGA_F32 || s->k > 1)
-    if ((st = launch_unpermute(*s, Op, inv, gate, O, cs)) != MOGA_OK) return st;
+  if ((st = forward_after_route(s, L, gid, gate, Q, K, V, O, perm_out, offsets_out, w, cs)) != MOGA_OK) return st;
   const size_t T = (size_t)s->N * s->k;
   if (gid_out) MOGA_CUDA_OK(cudaMemcpyAsync(gid_out, gid, sizeof(int32_t) * s->B * T, cudaMemcpyDeviceToDevice, cs));
   if (gate_out) MOGA_CUDA_OK(cudaMemcpyAsync(gate_out, gate, sizeof(float) * s->B * T, cudaMemcpyDeviceToDevice, cs));
-  if (perm_out) MOGA_CUDA_OK(cudaMemcpyAsync(perm_out, perm, sizeof(int32_t) * s->B * T, cudaMemcpyDeviceToDevice, cs));
-  if (offsets_out) MOGA_CUDA_OK(cudaMemcpyAsync(offsets_out, offsets, sizeof(int32_t) * s->B * (s->M + 1), cudaMemcpyDeviceToDevice, cs));
   return MOGA_OK;
 }
+
+moga_status moga_forward_routed(const moga_shape* s, const int32_t* gid, const float* gate, const void* Q,
+                                const void* K, const void* V, void* O, int32_t* perm_out, int32_t* offsets_out,
+                                void* ws, size_t ws_bytes, void* stream) {
+  moga_status st;
+  if (!check_shape(s, &st)) return st;
+  if (s->N == 0) {
+    if (offsets_out)
+      MOGA_CUDA_OK(cudaMemsetAsync(offsets_out, 0, sizeof(int32_t) * s->B * (s->M + 1), static_cast<cudaStream_t>(stream)));
+    return MOGA_OK;
+  }
+  if (!PTR_OK(gid) || !PTR_OK(gate) || !PTR_OK(Q) || !PTR_OK(K) || !PTR_OK(V) || !PTR_OK(O)) return MOGA_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(*s);
+  if (!check_ws(ws, ws_bytes, L.total, &st)) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  char* w = static_cast<char*>(ws);
+  if ((st = clear_header(w, L, cs)) != MOGA_OK) return st;
+  return forward_after_route(s, L, gid, gate, Q, K, V, O, perm_out, offsets_out, w, cs);
+}
+
+}  // extern "C"
+
+extern "C" {
 
 // ---- the whole visual-attention block (Sec. 3.2): routed branch + two static branches + mean
 namespace {
@@ -298,7 +339,7 @@ VisualLayout visual_layout(const moga_shape& s, int G, int Tkv, int F) {
   v.fr_scratch = take(moga_static_scratch_bytes(&s, F));
   v.fr_off = take(sizeof(int32_t) * ((size_t)F + 1));
   v.A = take(row * s.N);
-  v.C = take(row * s.N);
+  v.C = take(s.dtype == MOGA_BF16 && s.D == 128 ? 0 : row * s.N);   // the fused path never stores the third branch
   v.Qs = take(row * s.N);
   v.Ks = take(row * Tkv);
   v.Vs = take(row * Tkv);
@@ -330,23 +371,46 @@ moga_status moga_visual_forward(const moga_shape* s, const void* X, const float*
   if (!check_ws(ws, ws_bytes, v.total, &st)) return st;
   char* w = static_cast<char*>(ws);
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  // routed branch -> A
+  uint32_t* header = reinterpret_cast<uint32_t*>(w);   // == the routed branch's header: all launches report here
+  // routed branch -> A (clears the status header)
   st = moga_forward(s, X, Wr, bias, Q, K, V, w + v.A, nullptr, nullptr, nullptr, nullptr, w + v.fwd,
                     ws_layout(*s).total, stream);
   if (st != MOGA_OK) return st;
-  // spatial-temporal branch -> Bs (query order of the lists)
+  // spatial-temporal branch: gather by the lists, attention
   if ((st = launch_gather_list(*s, lists->q_idx, s->N, Q, w + v.Qs, cs)) != MOGA_OK) return st;
   if ((st = launch_gather_list(*s, lists->kv_idx, lists->Tkv, K, w + v.Ks, cs)) != MOGA_OK) return st;
   if ((st = launch_gather_list(*s, lists->kv_idx, lists->Tkv, V, w + v.Vs, cs)) != MOGA_OK) return st;
-  st = moga_static_group_attn(s, lists->G, s->N, lists->Tkv, w + v.Qs, w + v.Ks, w + v.Vs, lists->q_offsets,
-                              lists->kv_offsets, w + v.Bs, nullptr, w + v.st_scratch,
-                              moga_static_scratch_bytes(s, lists->G), stream);
-  if (st != MOGA_OK) return st;
-  // per-frame branch -> C (token order: a frame's tokens are contiguous)
   int32_t* fr_off = reinterpret_cast<int32_t*>(w + v.fr_off);
   if ((st = launch_frame_offsets(fr_off, lists->F, lists->tokens_per_frame, cs)) != MOGA_OK) return st;
-  st = moga_static_group_attn(s, lists->F, s->N, s->N, Q, K, V, fr_off, fr_off, w + v.C, nullptr, w + v.fr_scratch,
-                              moga_static_scratch_bytes(s, lists->F), stream);
+  if (s->dtype == MOGA_BF16 && s->D == 128) {
+    // tensor-core path: the spatial-temporal launch writes its rows straight to token order (Bs is
+    // then [B, H, N, D] in token order), and the per-frame launch, whose groups are contiguous
+    // frames, forms the mean of the three branches in its epilogue: no third tensor, no mean pass
+    st = launch_attn_bf16_static(*s, lists->G, s->N, lists->Tkv, w + v.Qs, w + v.Ks, w + v.Vs, lists->q_offsets,
+                                 lists->kv_offsets, w + v.Bs, nullptr, header, w + v.st_scratch + 256,
+                                 StaticEpilogue{lists->q_idx, nullptr, nullptr}, cs);
+    if (st != MOGA_OK) return st;
+    return launch_attn_bf16_static(*s, lists->F, s->N, s->N, Q, K, V, fr_off, fr_off, O, nullptr, header,
+                                   w + v.fr_scratch + 256, StaticEpilogue{nullptr, w + v.A, w + v.Bs}, cs);
+  }
+  // other types: the three branches are materialised and averaged by a separate pass
+  if (s->dtype == MOGA_BF16) {
+    st = launch_attn_bf16_static(*s, lists->G, s->N, lists->Tkv, w + v.Qs, w + v.Ks, w + v.Vs, lists->q_offsets,
+                                 lists->kv_offsets, w + v.Bs, nullptr, header, w + v.st_scratch + 256,
+                                 StaticEpilogue{nullptr, nullptr, nullptr}, cs);
+    if (st != MOGA_OK) return st;
+    st = launch_attn_bf16_static(*s, lists->F, s->N, s->N, Q, K, V, fr_off, fr_off, w + v.C, nullptr, header,
+                                 w + v.fr_scratch + 256, StaticEpilogue{nullptr, nullptr, nullptr}, cs);
+  } else {
+    st = launch_attn_f32_groups(s->B, s->H, s->D, s->scale, lists->G, s->N, lists->Tkv,
+                                reinterpret_cast<const float*>(w + v.Qs), reinterpret_cast<const float*>(w + v.Ks),
+                                reinterpret_cast<const float*>(w + v.Vs), lists->q_offsets, lists->kv_offsets, 0,
+                                reinterpret_cast<float*>(w + v.Bs), nullptr, cs);
+    if (st != MOGA_OK) return st;
+    st = launch_attn_f32_groups(s->B, s->H, s->D, s->scale, lists->F, s->N, s->N, static_cast<const float*>(Q),
+                                static_cast<const float*>(K), static_cast<const float*>(V), fr_off, fr_off, 0,
+                                reinterpret_cast<float*>(w + v.C), nullptr, cs);
+  }
   if (st != MOGA_OK) return st;
   return launch_mean3(*s, w + v.A, w + v.Bs, lists->q_inv, w + v.C, O, cs);
 }

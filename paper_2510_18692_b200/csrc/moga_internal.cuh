@@ -107,10 +107,20 @@ moga_status launch_attn_bf16_scatter(const moga_shape& s, const WsLayout& L, con
                                      const float* gate, void* O, char* ws, cudaStream_t st);
 
 // Static groups (Sec. 3.2): attention with caller-given query / key ranges per group, shared by
-// all batch items; ws holds the status header (256 B) and the schedule (2*B*G + 1 int32).
+// all batch items.  header: the device status word the kernel reports into (not cleared here);
+// sched: 2*B*G + 1 int32 of schedule scratch.  The epilogue either stores the rows in the order
+// of the query list (both pointers null), sends row p to token token_list[p] of a contiguous
+// [B, H, N, D] output, or (rows already in token order) stores the mean of the row and the rows
+// of mean_a and mean_b at the same place.  The last two need d_head = 128.
+struct StaticEpilogue {
+  const int32_t* token_list;
+  const void* mean_a;
+  const void* mean_b;
+};
 moga_status launch_attn_bf16_static(const moga_shape& s, int G, long long Tq, long long Tkv, const void* Qs,
                                     const void* Ks, const void* Vs, const int32_t* q_offsets,
-                                    const int32_t* kv_offsets, void* Os, float* lse, char* ws, cudaStream_t st);
+                                    const int32_t* kv_offsets, void* Os, float* lse, uint32_t* header, char* sched,
+                                    const StaticEpilogue& epi, cudaStream_t st);
 moga_status launch_attn_f32_groups(int B, int H, int D, float scale, int G, int Tq, int Tkv, const float* Qp,
                                    const float* Kp, const float* Vp, const int32_t* q_offsets,
                                    const int32_t* kv_offsets, int off_stride, float* Op, float* lse,

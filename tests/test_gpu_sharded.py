@@ -65,3 +65,32 @@ def test_shards_reproduce_the_unsharded_stages(mb):
         mb.moga_unpermute(sh, Op, inv, gate, Oh)
         torch.cuda.synchronize()
         assert torch.equal(offs, offsets) and torch.equal(Oh, O[:, lo:hi])
+
+
+@pytest.mark.parametrize("k,gate_mode", [(1, 0), (2, GATE_SOFTMAX_TOPK)])
+def test_forward_from_a_given_routing_is_the_forward(mb, k, gate_mode):
+    """moga_forward_routed fed with the routing moga_forward computed gives moga_forward's bits
+    (same kernels, the fused epilogue included), for all heads and for a head shard."""
+    cfg = MogaConfig("fr", 1, 4, 3001, 256, 128, 8, k, "bf16", gate_mode, 43)
+    inp = make_inputs(cfg, device="cuda")
+    sh = mb.make_shape(cfg)
+    ws = mb.alloc_workspace(mb.moga_workspace_bytes(sh))
+    O = torch.empty_like(inp["Q"])
+    gid = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.int32, device="cuda")
+    gate = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.float32, device="cuda")
+    offsets = torch.empty(cfg.B, cfg.M + 1, dtype=torch.int32, device="cuda")
+    mb.moga_forward(sh, inp["X"], inp["Wr"], inp["bias"], inp["Q"], inp["K"], inp["V"], O, ws, gid, gate, None, offsets)
+    assert mb.moga_last_device_status(ws) == (0, 0)
+    O2 = torch.full_like(O, float("nan"))
+    off2 = torch.empty_like(offsets)
+    mb.moga_forward_routed(sh, gid, gate, inp["Q"], inp["K"], inp["V"], O2, ws, None, off2)
+    assert mb.moga_last_device_status(ws) == (0, 0)
+    assert torch.equal(O2, O) and torch.equal(off2, offsets)
+    cfg_h = cfg.with_(H=1)
+    sh_h = mb.make_shape(cfg_h)
+    ws_h = mb.alloc_workspace(mb.moga_workspace_bytes(sh_h))
+    Qh, Kh, Vh = (inp[n][:, 2:3].contiguous() for n in ("Q", "K", "V"))
+    Oh = torch.empty_like(Qh)
+    mb.moga_forward_routed(sh_h, gid, gate, Qh, Kh, Vh, Oh, ws_h)
+    assert mb.moga_last_device_status(ws_h) == (0, 0)
+    assert torch.equal(Oh, O[:, 2:3])
