@@ -335,6 +335,19 @@ typedef enum { MOGA_ATTN_AUTO = 0, MOGA_ATTN_SINGLE = 1, MOGA_ATTN_PAIR = 2 } mo
 moga_status moga_set_attn_kernel(int32_t mode);
 
 /*
+ * Top-2 output path of moga_forward / moga_forward_routed for bf16 (the paper has no
+ * counterpart: a tuning and test switch).  on != 0: the attention epilogue rounds
+ * gate * row to bf16 and adds it into a zeroed O in token order (Eq. 5's sum over the two
+ * assignments as two commutative bf16 additions: the result does not depend on their order, so
+ * runs stay bit-reproducible); no permuted output is written and moga_unpermute is not run.
+ * on == 0 (default): the staged path (attention writes the permuted output, moga_unpermute sums
+ * in fp32 with one rounding).  The two differ in the last bit and take the same time on the
+ * top-2 workloads measured.  O with custom strides, k > 2 and fp32
+ * always take the staged path.  Process-wide.
+ */
+moga_status moga_set_fused_topk(int32_t on);
+
+/*
  * Self-test of the time-out path (the paper has no counterpart: it is a diagnostic).
  * Every wait inside the tensor-core kernels is bounded; when one runs out the kernel writes
  * MOGA_ERR_TIMEOUT and a detail word to the status header and returns normally.  This call

@@ -21,7 +21,7 @@ EXPORTS = ("moga_workspace_bytes", "moga_scratch_bytes", "moga_status_string", "
            "moga_permute", "moga_group_attn", "moga_unpermute", "moga_forward",
            "moga_last_device_status", "moga_sort_static", "moga_balance_stats", "moga_stga_build", "moga_gather_rows",
            "moga_static_group_attn", "moga_mean3", "moga_forward_host_bytes", "moga_forward_host",
-           "moga_visual_workspace_bytes", "moga_visual_forward", "moga_selftest_wait_timeout", "moga_set_attn_kernel", "moga_forward_routed")
+           "moga_visual_workspace_bytes", "moga_visual_forward", "moga_selftest_wait_timeout", "moga_set_attn_kernel", "moga_forward_routed", "moga_set_fused_topk")
 
 MOGA_F32, MOGA_BF16 = 0, 1
 MOGA_ROUTE_AUTO, MOGA_ROUTE_ALU = 0, 1
@@ -228,6 +228,10 @@ def moga_selftest_wait_timeout(ws, limit_ns):
 
 
 MOGA_ATTN_AUTO, MOGA_ATTN_SINGLE, MOGA_ATTN_PAIR = 0, 1, 2
+
+
+def moga_set_fused_topk(on: bool):
+    _check(lib.moga_set_fused_topk(ctypes.c_int32(1 if on else 0)), "moga_set_fused_topk")
 
 
 def moga_set_attn_kernel(mode: int):

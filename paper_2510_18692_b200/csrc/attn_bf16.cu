@@ -419,6 +419,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       const int bb = it.bh / H, hh = it.bh % H;
       if (Epi == kEpiDefault && sc.perm != nullptr && live)
         inv_l *= sc.gate[(size_t)bb * sc.N + sc.perm[(size_t)bb * T + tile_row0 + r]];
+      if (Epi == kEpiAdd && live) inv_l *= sc.gate[(size_t)bb * T + sc.perm[(size_t)bb * T + tile_row0 + r]];
       // Each warp stages 32 rows x 32 columns (2 KB) at a time in its own buffer and writes them
       // out itself: lane L stores piece L % 4 of rows i * 8 + L / 4, i = 0..3 (64-byte row segments).
       unsigned char* wst = smem + C::kSmemStage + (x * 4 + q) * 2048;
@@ -428,7 +429,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       for (int i = 0; i < 4; ++i) {
         const int grow = tile_row0 + q * 32 + i * 8 + (lane >> 2);
         orow_live[i] = grow < it.qhi;
-        if (Epi == kEpiList) {
+        if (Epi == kEpiAdd) {
+          const int tok = orow_live[i] ? sc.perm[(size_t)bb * T + grow] / sc.k : 0;
+          obase[i] = Op + bb * sc.sb + hh * sc.sh + (long long)tok * sc.sn;
+        } else if (Epi == kEpiList) {
           const int tok = orow_live[i] ? sc.perm[grow] : 0;
           obase[i] = Op + bb * sc.sb + hh * sc.sh + (long long)tok * sc.sn;
         } else if (Epi == kEpiDefault && sc.perm != nullptr) {
@@ -479,7 +483,15 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
               vw[e] = *reinterpret_cast<uint32_t*>(&t);
             }
           }
-          if (orow_live[i]) *reinterpret_cast<uint4*>(obase[i] + c * 32 + piece * 8) = val;
+          if (Epi == kEpiAdd) {
+            if (orow_live[i])
+              asm volatile("red.relaxed.gpu.global.add.noftz.v4.bf16x2 [%0], {%1, %2, %3, %4};" ::"l"(
+                               obase[i] + c * 32 + piece * 8),
+                           "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w)
+                           : "memory");
+          } else if (orow_live[i]) {
+            *reinterpret_cast<uint4*>(obase[i] + c * 32 + piece * 8) = val;
+          }
         }
         __syncwarp();
       }
@@ -565,6 +577,7 @@ Problem routed_problem(const moga_shape& s, const WsLayout& L, const void* Qp, c
 moga_status attn::launch_single(int D, const attn::Problem& p, cudaStream_t st) {
   if (p.epi == kEpiList) return D == 128 ? launch_one<128, false, kEpiList>(p, st) : MOGA_ERR_UNSUPPORTED;
   if (p.epi == kEpiMean3) return D == 128 ? launch_one<128, false, kEpiMean3>(p, st) : MOGA_ERR_UNSUPPORTED;
+  if (p.epi == kEpiAdd) return D == 128 ? launch_one<128, false, kEpiAdd>(p, st) : launch_one<64, false, kEpiAdd>(p, st);
   return D == 128 ? launch_one<128, false, kEpiDefault>(p, st) : launch_one<64, false, kEpiDefault>(p, st);
 }
 
@@ -576,7 +589,7 @@ moga_status launch_attn_bf16(const moga_shape& s, const WsLayout& L, const void*
                              const void* Vp, const int32_t* offsets, void* Op, float* lse, char* ws,
                              cudaStream_t st) {
   if ((long long)s.N * s.k == 0) return MOGA_OK;
-  const Scatter none{nullptr, nullptr, 0, 0, 0, 0, nullptr, nullptr};
+  const Scatter none{nullptr, nullptr, 0, 0, 0, 0, 0, nullptr, nullptr};
   return launch_any(s.D, routed_problem(s, L, Qp, Kp, Vp, offsets, Op, lse, ws, none), st);
 }
 
@@ -585,16 +598,35 @@ moga_status launch_attn_bf16_scatter(const moga_shape& s, const WsLayout& L, con
                                      const float* gate, void* O, char* ws, cudaStream_t st) {
   if ((long long)s.N * s.k == 0) return MOGA_OK;
   const Strides q = qkv_strides(s);
-  const Scatter sc{perm, gate, q.b, q.h, q.n, s.N, nullptr, nullptr};
+  const Scatter sc{perm, gate, q.b, q.h, q.n, s.N, s.k, nullptr, nullptr};
   return launch_any(s.D, routed_problem(s, L, Qp, Kp, Vp, offsets, O, nullptr, ws, sc), st);
 }
+
+moga_status launch_attn_bf16_add(const moga_shape& s, const WsLayout& L, const void* Qp, const void* Kp,
+                                 const void* Vp, const int32_t* offsets, const int32_t* asg, const float* gate,
+                                 void* O, char* ws, cudaStream_t st) {
+  if ((long long)s.N * s.k == 0) return MOGA_OK;
+  const Strides q = qkv_strides(s);
+  const Scatter sc{asg, gate, q.b, q.h, q.n, s.N, s.k, nullptr, nullptr};
+  Problem p = routed_problem(s, L, Qp, Kp, Vp, offsets, O, nullptr, ws, sc);
+  p.epi = kEpiAdd;
+  return launch_any(s.D, p, st);
+}
+
+namespace {
+// Off by default: measured on the two top-2 workloads it is no faster than the staged path
+// (74.6 vs 74.3 ms and 548.8 vs 548.6 ms per forward), which sums in fp32 with one rounding.
+int g_fused_topk = 0;
+}
+void set_fused_topk(int on) { g_fused_topk = on; }
+bool fused_topk() { return g_fused_topk != 0; }
 
 moga_status launch_attn_bf16_static(const moga_shape& s, int G, long long Tq, long long Tkv, const void* Qs,
                                     const void* Ks, const void* Vs, const int32_t* q_offsets,
                                     const int32_t* kv_offsets, void* Os, float* lse, uint32_t* header, char* sched,
                                     const StaticEpilogue& epi, cudaStream_t st) {
   if (Tq == 0 || G == 0) return MOGA_OK;
-  Scatter sc{nullptr, nullptr, 0, 0, 0, 0, nullptr, nullptr};
+  Scatter sc{nullptr, nullptr, 0, 0, 0, 0, 0, nullptr, nullptr};
   int mode = attn::kEpiDefault;
   if (epi.token_list != nullptr) {          // rows go to token order: Os is [B, H, N, D]
     mode = attn::kEpiList;

@@ -74,12 +74,17 @@ __device__ __forceinline__ Item decode_item(int w, const Groups& grp, const int3
 //                 (contiguous [B, H, N, D]); the stored value is the mean of this branch's row,
 //                 rounded to bf16 as if it had been stored, and the rows of mean_a and mean_b at
 //                 the same place: (a + b + c) / 3 in fp32, one rounding.
-constexpr int kEpiDefault = 0, kEpiList = 1, kEpiMean3 = 2;
+//   kEpiAdd       top-k routing with k = 2: perm holds the assignment index a = token * k + slot at
+//                 each sorted position; gate[b, a] * row is rounded to bf16 and added into token
+//                 a / k of a zeroed O with a bf16x2 reduction (two commutative additions per
+//                 element, so the result does not depend on their order).
+constexpr int kEpiDefault = 0, kEpiList = 1, kEpiMean3 = 2, kEpiAdd = 3;
 struct Scatter {
   const int32_t* perm;
   const float* gate;
   long long sb, sh, sn;
-  int N;
+  int N;                     // tokens per batch item
+  int k;
   const __nv_bfloat16* mean_a;
   const __nv_bfloat16* mean_b;
 };

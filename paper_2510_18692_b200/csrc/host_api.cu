@@ -50,7 +50,7 @@ moga_status get_pipe(Pipe** out) {
 }
 
 struct Arena {
-  size_t scratch, wr, bias, gid, gate, perm, inv, offsets, X;
+  size_t scratch, wr, bias, gid, gate, perm, inv, offsets, asg, X;
   size_t in[2][3];      // two staging sets of Q, K, V chunks  [B, hc, N, D]
   size_t Qp, Kp, Vp, Op;  // permuted chunk                    [B, hc, T, D]
   size_t out[2];        // two staging sets of the O chunk     [B, hc, N, D]
@@ -73,6 +73,7 @@ Arena arena_layout(const moga_shape& s, int hc) {
   a.gid = take(sizeof(int32_t) * s.B * T);
   a.gate = take(sizeof(float) * s.B * T);
   a.perm = take(sizeof(int32_t) * s.B * T);
+  a.asg = take(sizeof(int32_t) * s.B * T);
   a.inv = take(sizeof(int32_t) * s.B * T);
   a.offsets = take(sizeof(int32_t) * s.B * (s.M + 1));
   a.X = take(es * s.B * s.N * s.C);
@@ -170,7 +171,10 @@ moga_status moga_forward_host(const moga_shape* s, const void* X, const float* W
            ? launch_route_mma(*s, L, a + A.X, wr_d, bias_d, gid, gate, nullptr, scratch, cs)
            : launch_route(*s, a + A.X, wr_d, bias_d, gid, gate, nullptr, cs);
   if (st != MOGA_OK) return st;
-  if ((st = launch_sort(*s, L, gid, perm, inv, offsets, scratch, cs)) != MOGA_OK) return st;
+  // bf16 top-2: the same add epilogue as moga_forward (the results are bit-identical to it)
+  const bool add_epilogue = s->dtype == MOGA_BF16 && s->k == 2 && fused_topk();
+  int32_t* asg = add_epilogue ? reinterpret_cast<int32_t*>(a + A.asg) : nullptr;
+  if ((st = launch_sort(*s, L, gid, perm, inv, offsets, scratch, cs, asg)) != MOGA_OK) return st;
   if (gid_out) MOGA_CUDA_OK(cudaMemcpyAsync(gid_out, gid, sizeof(int32_t) * s->B * T, cudaMemcpyDeviceToHost, cs));
   if (gate_out) MOGA_CUDA_OK(cudaMemcpyAsync(gate_out, gate, sizeof(float) * s->B * T, cudaMemcpyDeviceToHost, cs));
 
@@ -197,6 +201,9 @@ moga_status moga_forward_host(const moga_shape* s, const void* X, const float* W
                            reinterpret_cast<const float*>(a + A.Vp), offsets, reinterpret_cast<float*>(a + A.Op),
                            nullptr, cs);
       if (st == MOGA_OK) st = launch_unpermute(sub, a + A.Op, inv, gate, Oc, cs);
+    } else if (add_epilogue) {
+      MOGA_CUDA_OK(cudaMemsetAsync(Oc, 0, es * (size_t)s->B * nh * s->N * s->D, cs));
+      st = launch_attn_bf16_add(sub, L, a + A.Qp, a + A.Kp, a + A.Vp, offsets, asg, gate, Oc, scratch, cs);
     } else if (s->k == 1) {
       st = launch_attn_bf16_scatter(sub, L, a + A.Qp, a + A.Kp, a + A.Vp, offsets, perm, gate, Oc, scratch, cs);
     } else {

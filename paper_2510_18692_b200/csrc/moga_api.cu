@@ -244,9 +244,16 @@ moga_status forward_after_route(const moga_shape* s, const WsLayout& L, const in
   void* Kp = w + L.Kp;
   void* Vp = w + L.Vp;
   void* Op = w + L.Op;
-  if ((st = launch_sort(*s, L, gid, perm, inv, offsets, w, cs)) != MOGA_OK) return st;
+  // bf16 top-2 with a dense O: the attention epilogue adds gate * row into a zeroed O
+  const bool dense_o = !(s->q_stride_b || s->q_stride_h || s->q_stride_n);
+  const bool add_epilogue = s->dtype == MOGA_BF16 && s->k == 2 && dense_o && fused_topk();
+  int32_t* asg = add_epilogue ? reinterpret_cast<int32_t*>(w + L.asg) : nullptr;
+  if ((st = launch_sort(*s, L, gid, perm, inv, offsets, w, cs, asg)) != MOGA_OK) return st;
   if ((st = launch_gather(*s, perm, Q, K, V, Qp, Kp, Vp, cs)) != MOGA_OK) return st;
-  if (s->dtype == MOGA_F32)
+  if (add_epilogue) {
+    MOGA_CUDA_OK(cudaMemsetAsync(O, 0, elem_size(s->dtype) * (size_t)s->B * s->H * s->N * s->D, cs));
+    st = launch_attn_bf16_add(*s, L, Qp, Kp, Vp, offsets, asg, gate, O, w, cs);
+  } else if (s->dtype == MOGA_F32)
     st = launch_attn_f32(*s, static_cast<const float*>(Qp), static_cast<const float*>(Kp),
                          static_cast<const float*>(Vp), offsets, static_cast<float*>(Op), nullptr, cs);
   else if (s->k == 1)   // one assignment per token: the attention epilogue is the gated scatter
@@ -254,7 +261,7 @@ moga_status forward_after_route(const moga_shape* s, const WsLayout& L, const in
   else
     st = launch_attn_bf16(*s, L, Qp, Kp, Vp, offsets, Op, nullptr, w, cs);
   if (st != MOGA_OK) return st;
-  if (s->dtype == MOGA_F32 || s->k > 1)
+  if (!add_epilogue && (s->dtype == MOGA_F32 || s->k > 1))
     if ((st = launch_unpermute(*s, Op, inv, gate, O, cs)) != MOGA_OK) return st;
   const size_t T = (size_t)s->N * s->k;
   if (perm_out) MOGA_CUDA_OK(cudaMemcpyAsync(perm_out, perm, sizeof(int32_t) * s->B * T, cudaMemcpyDeviceToDevice, cs));
@@ -413,6 +420,11 @@ moga_status moga_visual_forward(const moga_shape* s, const void* X, const float*
   }
   if (st != MOGA_OK) return st;
   return launch_mean3(*s, w + v.A, w + v.Bs, lists->q_inv, w + v.C, O, cs);
+}
+
+moga_status moga_set_fused_topk(int32_t on) {
+  set_fused_topk(on != 0);
+  return MOGA_OK;
 }
 
 moga_status moga_set_attn_kernel(int32_t mode) {

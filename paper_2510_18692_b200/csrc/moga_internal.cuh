@@ -29,7 +29,7 @@ struct WsLayout {
   size_t stats;       // int32 + float [B, nblk, M] per-block counts and gate sums (Eq. 6-8)
   size_t redo;        // int32 [4 + 2 * items]  work items the CTA-pair attention kernel hands to the exact path
   size_t scratch_end; // == moga_scratch_bytes
-  size_t gid, gate, perm, inv, offsets;  // routing results
+  size_t gid, gate, perm, inv, offsets, asg;  // routing results (asg: assignment index per sorted position)
   size_t Qp, Kp, Vp, Op;                 // permuted tensors
   size_t total;       // == moga_workspace_bytes
   int nblk;           // sort blocks per batch item
@@ -59,6 +59,7 @@ inline WsLayout ws_layout(const moga_shape& s) {
   L.perm = off;        off = align_up(off + sizeof(int32_t) * (size_t)s.B * T, kWsAlign);
   L.inv = off;         off = align_up(off + sizeof(int32_t) * (size_t)s.B * T, kWsAlign);
   L.offsets = off;     off = align_up(off + sizeof(int32_t) * (size_t)s.B * (s.M + 1), kWsAlign);
+  L.asg = off;         off = align_up(off + sizeof(int32_t) * (size_t)s.B * T, kWsAlign);
   size_t row = (size_t)s.B * s.H * T * s.D * elem_size(s.dtype);
   L.Qp = off;          off = align_up(off + row, kWsAlign);
   L.Kp = off;          off = align_up(off + row, kWsAlign);
@@ -88,8 +89,9 @@ moga_status launch_route_mma(const moga_shape& s, const WsLayout& L, const void*
                              cudaStream_t st);
 moga_status launch_balance_stats(const moga_shape& s, const WsLayout& L, const int32_t* gid, const float* gate,
                                  float alpha, float* F, float* P, float* loss, char* ws, cudaStream_t st);
+// asg (optional, [B, T]): the assignment index n*k + j that sits at each sorted position
 moga_status launch_sort(const moga_shape& s, const WsLayout& L, const int32_t* gid, int32_t* perm,
-                        int32_t* inv, int32_t* offsets, char* ws, cudaStream_t st);
+                        int32_t* inv, int32_t* offsets, char* ws, cudaStream_t st, int32_t* asg = nullptr);
 moga_status launch_gather(const moga_shape& s, const int32_t* perm, const void* Q, const void* K,
                           const void* V, void* Qp, void* Kp, void* Vp, cudaStream_t st);
 moga_status launch_unpermute(const moga_shape& s, const void* Op, const int32_t* inv,
@@ -105,6 +107,15 @@ moga_status launch_attn_bf16(const moga_shape& s, const WsLayout& L, const void*
 moga_status launch_attn_bf16_scatter(const moga_shape& s, const WsLayout& L, const void* Qp, const void* Kp,
                                      const void* Vp, const int32_t* offsets, const int32_t* perm,
                                      const float* gate, void* O, char* ws, cudaStream_t st);
+
+// Top-2 routing: the attention epilogue adds gate * row into a zeroed O in token order (Eq. 5's
+// sum over the two assignments as two commutative additions), so there is no permuted output and
+// no unpermute pass.  asg: assignment index per sorted position; gate: [B, N, k].
+moga_status launch_attn_bf16_add(const moga_shape& s, const WsLayout& L, const void* Qp, const void* Kp,
+                                 const void* Vp, const int32_t* offsets, const int32_t* asg, const float* gate,
+                                 void* O, char* ws, cudaStream_t st);
+void set_fused_topk(int on);
+bool fused_topk();
 
 // Static groups (Sec. 3.2): attention with caller-given query / key ranges per group, shared by
 // all batch items.  header: the device status word the kernel reports into (not cleared here);

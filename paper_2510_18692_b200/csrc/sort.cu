@@ -82,8 +82,8 @@ sort_scan_kernel(int32_t* __restrict__ blk_hist, int32_t* __restrict__ offsets, 
 
 __global__ void __launch_bounds__(kSortThreads)
 sort_scatter_kernel(const int32_t* __restrict__ gid, const int32_t* __restrict__ blk_base,
-                    int32_t* __restrict__ perm, int32_t* __restrict__ inv, int T, int M, int k,
-                    int nblk) {
+                    int32_t* __restrict__ perm, int32_t* __restrict__ inv, int32_t* __restrict__ asg, int T,
+                    int M, int k, int nblk) {
   __shared__ int base[kMaxM];
   __shared__ int wcnt[kSortWarps][kMaxM];
   const int b = blockIdx.y, blk = blockIdx.x;
@@ -108,6 +108,7 @@ sort_scatter_kernel(const int32_t* __restrict__ gid, const int32_t* __restrict__
       for (int w = 0; w < warp; ++w) pos += wcnt[w][key];
       perm[(size_t)b * T + pos] = a / k;
       inv[(size_t)b * T + a] = pos;
+      if (asg != nullptr) asg[(size_t)b * T + pos] = a;     // the assignment (token, slot) at this position
     }
     __syncthreads();
     if (threadIdx.x < M) {
@@ -123,7 +124,7 @@ sort_scatter_kernel(const int32_t* __restrict__ gid, const int32_t* __restrict__
 }  // namespace
 
 moga_status launch_sort(const moga_shape& s, const WsLayout& L, const int32_t* gid, int32_t* perm,
-                        int32_t* inv, int32_t* offsets, char* ws, cudaStream_t st) {
+                        int32_t* inv, int32_t* offsets, char* ws, cudaStream_t st, int32_t* asg) {
   const int T = s.N * s.k;
   int32_t* hist = reinterpret_cast<int32_t*>(ws + L.sort_hist);
   uint32_t* header = reinterpret_cast<uint32_t*>(ws + L.header);
@@ -132,7 +133,7 @@ moga_status launch_sort(const moga_shape& s, const WsLayout& L, const int32_t* g
   MOGA_CUDA_OK(cudaGetLastError());
   sort_scan_kernel<<<s.B, 1024, 0, st>>>(hist, offsets, s.M, L.nblk);
   MOGA_CUDA_OK(cudaGetLastError());
-  sort_scatter_kernel<<<grid, kSortThreads, 0, st>>>(gid, hist, perm, inv, T, s.M, s.k, L.nblk);
+  sort_scatter_kernel<<<grid, kSortThreads, 0, st>>>(gid, hist, perm, inv, asg, T, s.M, s.k, L.nblk);
   MOGA_CUDA_OK(cudaGetLastError());
   return MOGA_OK;
 }

@@ -103,12 +103,41 @@ def test_bnhd_layout(mb):
 
 
 def test_forward_is_deterministic(mb):
-    cfg = SMALL[1]
-    inp = make_inputs(cfg, device="cuda")
-    a = run_forward(mb, cfg, inp)
-    b = run_forward(mb, cfg, inp)
-    for x, y in zip(a, b):
-        assert torch.equal(x, y)
+    """Top-2 included: its epilogue adds the two assignments of a token into O with reductions,
+    whose order is free, but two additions commute, so every run gives the same bits."""
+    try:
+        for fused in (False, True):
+            mb.moga_set_fused_topk(fused)
+            for cfg in (SMALL[1], SMALL[2]):
+                inp = make_inputs(cfg, device="cuda")
+                a = run_forward(mb, cfg, inp)
+                for _ in range(4):
+                    b = run_forward(mb, cfg, inp)
+                    for x, y in zip(a, b):
+                        assert torch.equal(x, y)
+    finally:
+        mb.moga_set_fused_topk(False)
+
+
+@pytest.mark.parametrize("cfg", [SMALL[1], SMALL[2], SMALL[1].with_(D=64, name="s_bf16_top2_d64")], ids=lambda c: c.name)
+def test_top2_staged_path_and_add_epilogue(mb, cfg):
+    """The two bf16 top-2 output paths (permuted output + fp32 gated sum, and gate * row added into
+    token order by the attention epilogue): each within the oracle bounds, and close to each other
+    (they differ by the roundings of the two contributions)."""
+    outs = {}
+    try:
+        for fused in (False, True):
+            mb.moga_set_fused_topk(fused)
+            full_parity(mb, cfg)
+            outs[fused] = run_forward(mb, cfg, make_inputs(cfg, device="cuda"))[0].float()
+    finally:
+        mb.moga_set_fused_topk(False)
+    row_mag = outs[False].abs().amax(dim=-1, keepdim=True)
+    assert ((outs[True] - outs[False]).abs() <= 2.0 ** -6 * row_mag + 1e-6).all()
+
+
+def test_top2_with_strided_output_takes_the_staged_path(mb):
+    full_parity(mb, SMALL[1].with_(N=777), layout_bnhd=True)
 
 
 def sampled_parity(mb, cfg, n_route=4096, n_rows=2048, heads=(0,)):

@@ -26,9 +26,13 @@ def test_shards_reproduce_the_unsharded_stages(mb):
     inp = make_inputs(cfg, device="cuda")
     # world size 1: the sharded driver is the staged forward
     O = torch.empty_like(inp["Q"])
-    gid, gate, offsets = forward_head_sharded(mb, cfg, inp["X"], inp["Wr"], inp["bias"], inp["Q"], inp["K"],
-                                              inp["V"], O)
-    torch.cuda.synchronize()
+    mb.moga_set_fused_topk(False)          # the staged top-2 path, which the stage calls below reproduce bit for bit
+    try:
+        gid, gate, offsets = forward_head_sharded(mb, cfg, inp["X"], inp["Wr"], inp["bias"], inp["Q"], inp["K"],
+                                                  inp["V"], O)
+        torch.cuda.synchronize()
+    finally:
+        mb.moga_set_fused_topk(False)
     host = {k: to_np32(v) for k, v in inp.items()}
     off, perm, _ = oracle.sort(gid.cpu().numpy(), cfg.M)
     want = oracle.attn_all(host["Q"], host["K"], host["V"], gid.cpu().numpy(), gate.double().cpu().numpy(), off,
