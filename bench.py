@@ -40,7 +40,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes of the attention kernel / its algorithmic bytes, from the ncu capture of the
 # clip-sized case (traffic grows with T*H: every Q/K/V/O byte crosses DRAM once).  The figure
 # belongs to one version of the kernel source: when the source's hash differs, traffic is null.
-ATTN_TRAFFIC = {"ratio": 0.958, "source_sha16": "@@SHA@@"}
+ATTN_TRAFFIC = {"ratio": 0.9565, "source_sha16": "6a7a8dee240eb5b1"}
 
 
 def attn_traffic_ratio():
@@ -52,6 +52,30 @@ def attn_traffic_ratio():
     except OSError:
         return None
     return ATTN_TRAFFIC["ratio"] if sha == ATTN_TRAFFIC["source_sha16"] else None
+
+
+def schedule_tail(offsets_np, H, n_ctas=148, qblock=256, tile_n=128):
+    """Imbalance of the attention kernel's static schedule for these group sizes: work items of
+    `qblock` query rows, groups in order of decreasing cost inside each batch item, item w goes to
+    CTA w mod n_ctas.  An item costs (query tiles) x (key tiles).  Returns max over CTAs of the
+    assigned cost / mean."""
+    load = np.zeros(n_ctas)
+    w = 0
+    for b in range(offsets_np.shape[0]):
+        sizes = np.diff(offsets_np[b]).astype(np.int64)
+        for g in np.argsort(-(sizes * sizes), kind="stable"):
+            n = int(sizes[g])
+            if n == 0:
+                continue
+            nqb, ktiles = -(-n // qblock), -(-n // tile_n)
+            last_rows = n - (nqb - 1) * qblock
+            costs = np.full(nqb, 2.0 * ktiles)
+            costs[-1] = (2.0 if last_rows > tile_n else 1.0) * ktiles
+            items = np.tile(costs, H)                 # head-major, query block fastest
+            idx = (w + np.arange(items.size)) % n_ctas
+            np.add.at(load, idx, items)
+            w += items.size
+    return float(load.max() / load.mean()) if load.mean() > 0 else 1.0
 
 
 def kernels_per_forward(cfg):
@@ -242,6 +266,12 @@ def main():
                     help="'route' times moga_route alone on the config's X (a small resident set, for profiling); "
                          "'visual' times the whole visual-attention block: routed branch, the two static-group "
                          "branches and their mean")
+    ap.add_argument("--attn-kernel", default="auto", choices=["auto", "single", "pair"],
+                    help="bf16 group-attention kernel (moga_set_attn_kernel): the one-CTA kernel (default) or the "
+                         "CTA-pair kernel, for A/B runs and profiles")
+    ap.add_argument("--topk-epilogue", default="staged", choices=["staged", "add"],
+                    help="bf16 top-2 output path (moga_set_fused_topk): permuted output + unpermute (default) or "
+                         "gate * row added into token order by the attention epilogue")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = CONFIGS[args.config]
@@ -259,6 +289,8 @@ def main():
     build.build()
     from paper_2510_18692_b200 import binding as mb   # raises if the CUDA library is missing
 
+    mb.moga_set_attn_kernel({"auto": 0, "single": 1, "pair": 2}[args.attn_kernel])
+    mb.moga_set_fused_topk(args.topk_epilogue == "add")
     cfg = cfg.with_(seed=cfg.seed + 100 * rank)       # every rank works on its own layer
     if args.sharding == "auto":
         args.sharding = "heads" if world > 1 else "layers"
@@ -367,9 +399,12 @@ def main():
         "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic", "config": config_dict(cfg),
         "route_kernel": "tensor" if cfg.dtype == "bf16" else "alu",
+        "attn_kernel": ("pair" if args.attn_kernel == "pair" and cfg.D == 128 else "single") if cfg.dtype == "bf16" else "alu",
+        "topk_epilogue": args.topk_epilogue if (cfg.dtype == "bf16" and cfg.k == 2) else None,
         "ms_per_layer_head_batch": ms / (cfg.B * cfg.H), "useful_tflop_per_step": flops / 1e12,
         "group_sizes": {"min": int(sizes.min()), "max": int(sizes.max()), "empty": int((sizes == 0).sum())},
         "stages": stages_out, "gpu_launches": kernels_per_forward(cfg) * args.steps, "clocks": clk,
+        "schedule_tail": schedule_tail(offsets.cpu().numpy(), cfg.H) if cfg.dtype == "bf16" else None,
     }
     if cfg.dtype == "bf16":
         out["roofline"] = {

@@ -51,6 +51,8 @@ class MogaConfig:
 # top-2 cases use a softmax over the two selected logits.
 CONFIGS = {
     "tiny_f32": MogaConfig("tiny_f32", 1, 2, 4096, 128, 64, 8, 1, "f32", GATE_SOFTMAX_ALL, 0),
+    # the same case with one group: MoGA must then equal full attention (gate = 1)
+    "tiny_f32_m1": MogaConfig("tiny_f32_m1", 1, 2, 4096, 128, 64, 1, 1, "f32", GATE_SOFTMAX_ALL, 0),
     "clip_bf16": MogaConfig("clip_bf16", 1, 12, 32760, 1536, 128, 8, 1, "bf16", GATE_SOFTMAX_ALL, 1),
     "multishot_bf16": MogaConfig("multishot_bf16", 1, 40, 126360, 5120, 128, 16, 2, "bf16",
                                  GATE_SOFTMAX_TOPK, 2),
