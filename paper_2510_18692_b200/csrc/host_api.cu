@@ -191,7 +191,7 @@ moga_status moga_forward_host(const moga_shape* s, const void* X, const float* W
     // compute
     MOGA_CUDA_OK(cudaStreamWaitEvent(cs, P->chunk_in[c], 0));
     if ((st = launch_gather(sub, perm, a + A.in[set][0], a + A.in[set][1], a + A.in[set][2], a + A.Qp, a + A.Kp,
-                            a + A.Vp, cs)) != MOGA_OK)
+                            a + A.Vp, cs, inv)) != MOGA_OK)
       return st;
     MOGA_CUDA_OK(cudaEventRecord(P->gathered[c], cs));
     if (c >= 2) MOGA_CUDA_OK(cudaStreamWaitEvent(cs, P->chunk_out[c - 2], 0));   // O staging set free again

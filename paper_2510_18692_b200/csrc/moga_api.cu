@@ -144,7 +144,7 @@ moga_status moga_permute(const moga_shape* s, const int32_t* gid, const void* Q,
   char* w = static_cast<char*>(ws);
   if ((st = clear_header(w, L, cs)) != MOGA_OK) return st;
   if ((st = launch_sort(*s, L, gid, perm, inv, offsets, w, cs)) != MOGA_OK) return st;
-  if (n_out == 3) return launch_gather(*s, perm, Q, K, V, Qp, Kp, Vp, cs);
+  if (n_out == 3) return launch_gather(*s, perm, Q, K, V, Qp, Kp, Vp, cs, inv);
   return MOGA_OK;
 }
 
@@ -249,7 +249,7 @@ moga_status forward_after_route(const moga_shape* s, const WsLayout& L, const in
   const bool add_epilogue = s->dtype == MOGA_BF16 && s->k == 2 && dense_o && fused_topk();
   int32_t* asg = add_epilogue ? reinterpret_cast<int32_t*>(w + L.asg) : nullptr;
   if ((st = launch_sort(*s, L, gid, perm, inv, offsets, w, cs, asg)) != MOGA_OK) return st;
-  if ((st = launch_gather(*s, perm, Q, K, V, Qp, Kp, Vp, cs)) != MOGA_OK) return st;
+  if ((st = launch_gather(*s, perm, Q, K, V, Qp, Kp, Vp, cs, inv)) != MOGA_OK) return st;
   if (add_epilogue) {
     MOGA_CUDA_OK(cudaMemsetAsync(O, 0, elem_size(s->dtype) * (size_t)s->B * s->H * s->N * s->D, cs));
     st = launch_attn_bf16_add(*s, L, Qp, Kp, Vp, offsets, asg, gate, O, w, cs);

@@ -92,8 +92,10 @@ moga_status launch_balance_stats(const moga_shape& s, const WsLayout& L, const i
 // asg (optional, [B, T]): the assignment index n*k + j that sits at each sorted position
 moga_status launch_sort(const moga_shape& s, const WsLayout& L, const int32_t* gid, int32_t* perm,
                         int32_t* inv, int32_t* offsets, char* ws, cudaStream_t st, int32_t* asg = nullptr);
+// inv (optional): with it and 2 <= k <= 4 the copy runs token by token (each row read once, written k times)
 moga_status launch_gather(const moga_shape& s, const int32_t* perm, const void* Q, const void* K,
-                          const void* V, void* Qp, void* Kp, void* Vp, cudaStream_t st);
+                          const void* V, void* Qp, void* Kp, void* Vp, cudaStream_t st,
+                          const int32_t* inv = nullptr);
 moga_status launch_unpermute(const moga_shape& s, const void* Op, const int32_t* inv,
                              const float* gate, void* O, cudaStream_t st);
 moga_status launch_attn_f32(const moga_shape& s, const float* Qp, const float* Kp, const float* Vp,
