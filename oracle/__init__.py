@@ -246,3 +246,50 @@ def static_group_attn_rows(Q, K, V, q_groups, kv_groups, scale, rows):
 def mean3(a, b, c):
     """Sec. 3.2: a token's output is the mean of its dynamic (MoGA) and two static group outputs."""
     return (np.asarray(a, np.float64) + np.asarray(b, np.float64) + np.asarray(c, np.float64)) / 3.0
+
+
+# ----------------------------------------------------------------------------- backward
+def backward(Q, K, V, gid, gate, dO, scale, M):
+    """Gradients of the routed group attention with respect to Q, K, V and the gates.
+
+    The paper states no backward pass; this is the chain rule applied to its forward definition,
+    O[b,h,n] = sum_j gate[b,n,j] * SA(q_n, K_g, V_g) with g = gid[b,n,j] (Eq. 5 around Eq. 1), for a
+    given upstream gradient dO = dL/dO, written out group by group in fp64 with dense matrices:
+      p = softmax(scale * q k^T) (rows), o = p v
+      do = gate * dO                      (gradient reaching the group's attention output)
+      dgate = sum over heads and channels of dO * o
+      dv = p^T do,  dp = do v^T,  ds = p * (dp - rowsum(dp * p)),  dq = scale * ds k,  dk = scale * ds^T q
+    A token routed to k groups receives the sum of its k contributions.  The routing (gid) is a
+    fixed integer decision and carries no gradient.
+    Q, K, V, dO [B,H,N,D]; gid int [B,N,k]; gate [B,N,k].  Returns dQ, dK, dV [B,H,N,D], dgate [B,N,k] (fp64)."""
+    Q, K, V, dO = (np.asarray(a, dtype=np.float64) for a in (Q, K, V, dO))
+    gid = np.asarray(gid)
+    gate = np.asarray(gate, dtype=np.float64)
+    B, H, N, D = Q.shape
+    k = gid.shape[2]
+    dQ, dK, dV = np.zeros_like(Q), np.zeros_like(K), np.zeros_like(V)
+    dgate = np.zeros((B, N, k))
+    for b in range(B):
+        for g in range(M):
+            tok, slot = np.nonzero(gid[b] == g)            # assignments of group g, ascending token
+            if tok.size == 0:
+                continue
+            gt = gate[b, tok, slot]
+            for h in range(H):
+                q, kk, v = Q[b, h, tok], K[b, h, tok], V[b, h, tok]
+                s = scale * (q @ kk.T)
+                s = s - s.max(axis=1, keepdims=True)
+                p = np.exp(s)
+                p /= p.sum(axis=1, keepdims=True)
+                o = p @ v
+                d_out = dO[b, h, tok]
+                np.add.at(dgate[b], (tok, slot), (d_out * o).sum(axis=1))
+                do = gt[:, None] * d_out
+                dv = p.T @ do
+                dp = do @ v.T
+                ds = p * (dp - (dp * p).sum(axis=1, keepdims=True))
+                np.add.at(dQ[b, h], tok, scale * (ds @ kk))
+                np.add.at(dK[b, h], tok, scale * (ds.T @ q))
+                np.add.at(dV[b, h], tok, dv)
+    return dQ, dK, dV, dgate
+

@@ -398,3 +398,72 @@ def test_static_group_attention_agrees_with_the_routed_oracle():
     a = oracle.static_group_attn(Q, K, V, groups, groups, 0.3)
     b = oracle.attn_all(Q, K, V, gid, np.ones((B, N, 1)), offsets, perm, 0.3)
     assert np.abs(a - b).max() < 1e-12
+
+
+# ----------------------------------------------------------------------------- backward
+def _torch_forward_masked(Q, K, V, gid, gate, scale):
+    """The forward of Eq. 1 + Eq. 5 written a different way (dense N x N scores with a same-group
+    mask per slot, torch fp64 ops), so that autograd gives gradients independent of the oracle."""
+    B, H, N, D = Q.shape
+    k = gid.shape[2]
+    O = torch.zeros_like(Q)
+    s = torch.einsum("bhnd,bhmd->bhnm", Q, K) * scale
+    for j in range(k):
+        # query n (slot j) may attend key m iff m is assigned, in any slot, to the group gid[n, j]
+        same = (gid[:, :, j][:, :, None, None] == gid[:, None, :, :]).any(-1)        # [B, N, N]
+        sj = s.masked_fill(~same[:, None], float("-inf"))
+        O = O + gate[:, None, :, j, None] * torch.einsum("bhnm,bhmd->bhnd", torch.softmax(sj, -1), V)
+    return O
+
+
+@pytest.mark.parametrize("k", [1, 2])
+def test_backward_oracle_against_autograd_and_finite_differences(k):
+    rng = np.random.default_rng(17 + k)
+    B, H, N, D, M = 2, 2, 37, 8, 4
+    Q, K, V, dO = (rng.standard_normal((B, H, N, D)) for _ in range(4))
+    gid = np.stack([rng.permutation(M)[:k] for _ in range(B * N)]).reshape(B, N, k).astype(np.int32)
+    gate = rng.random((B, N, k)) + 0.1
+    scale = 0.4
+    dQ, dK, dV, dgate = oracle.backward(Q, K, V, gid, gate, dO, scale, M)
+    tq, tk, tv, tg = (torch.tensor(a, dtype=torch.float64, requires_grad=True) for a in (Q, K, V, gate))
+    out = _torch_forward_masked(tq, tk, tv, torch.tensor(gid.astype(np.int64)), tg, scale)
+    # the masked torch forward is itself the oracle's forward
+    off, perm, _ = oracle.sort(gid, M)
+    want = oracle.attn_all(Q.astype(np.float32), K.astype(np.float32), V.astype(np.float32), gid, gate, off, perm, scale)
+    ref32 = _torch_forward_masked(*(torch.tensor(a.astype(np.float32).astype(np.float64)) for a in (Q, K, V)),
+                                  torch.tensor(gid.astype(np.int64)), torch.tensor(gate), scale)
+    assert np.abs(ref32.numpy() - want).max() < 1e-12
+    gq, gk, gv, gg = torch.autograd.grad(out, (tq, tk, tv, tg), torch.tensor(dO))
+    for mine, ref in ((dQ, gq), (dK, gk), (dV, gv), (dgate, gg)):
+        assert np.abs(mine - ref.numpy()).max() < 1e-11
+    # central differences of L = sum(dO * O) on a few coordinates
+    def loss(q, kk, v, g):
+        return float((dO * _torch_forward_masked(*(torch.tensor(a) for a in (q, kk, v)),
+                                                 torch.tensor(gid.astype(np.int64)), torch.tensor(g), scale).numpy()).sum())
+    eps = 1e-6
+    for arr, grad, name in ((Q, dQ, "q"), (K, dK, "k"), (V, dV, "v")):
+        idx = (1, 0, 5, 3)
+        hi, lo = arr.copy(), arr.copy()
+        hi[idx] += eps
+        lo[idx] -= eps
+        args = {"q": (hi, K, V), "k": (Q, hi, V), "v": (Q, K, hi)}[name], {"q": (lo, K, V), "k": (Q, lo, V), "v": (Q, K, lo)}[name]
+        fd = (loss(*args[0], gate) - loss(*args[1], gate)) / (2 * eps)
+        assert abs(fd - grad[idx]) < 1e-6 * max(1.0, abs(fd))
+
+
+def test_backward_oracle_special_cases():
+    """One-token groups: o = v, so dV = gate * dO, dQ = dK = 0, dgate = <dO, v>.  Equal V rows in a
+    group: the output does not depend on the scores, so dQ = dK = 0 there."""
+    rng = np.random.default_rng(3)
+    B, H, N, D, M = 1, 1, 6, 4, 6
+    Q, K, V, dO = (rng.standard_normal((B, H, N, D)) for _ in range(4))
+    gid = np.arange(N, dtype=np.int32).reshape(1, N, 1)          # every token alone in its group
+    gate = rng.random((1, N, 1)) + 0.5
+    dQ, dK, dV, dgate = oracle.backward(Q, K, V, gid, gate, dO, 0.7, M)
+    assert np.abs(dQ).max() == 0 and np.abs(dK).max() == 0
+    assert np.abs(dV - gate[:, None, :, 0, None] * dO).max() < 1e-15
+    assert np.abs(dgate[..., 0] - (dO * V).sum(-1)[:, 0]).max() < 1e-15
+    gid2 = np.zeros((1, N, 1), np.int32)
+    V2 = np.broadcast_to(V[:, :, :1], V.shape).copy()
+    dQ2, dK2, dV2, _ = oracle.backward(Q, K, V2, gid2, gate, dO, 0.7, 1)
+    assert np.abs(dQ2).max() < 1e-15 and np.abs(dK2).max() < 1e-15
