@@ -321,6 +321,28 @@ moga_status moga_forward_host(const moga_shape* s, const void* X, const float* W
 moga_status moga_last_device_status(void* ws, void* stream, uint32_t* detail);
 
 /*
+ * Backward of the routed group attention (the paper states no backward pass: this is the chain
+ * rule applied to Eq. 1 inside each group and the gate of Eq. 5; the routing decision carries no
+ * gradient).  bf16, d_head = 128 (else MOGA_ERR_UNSUPPORTED).
+ * Saved from a forward made of the stage calls, all in sorted order: Qp, Kp, Vp (moga_permute),
+ * Op and lse (moga_group_attn), [B, H, T, D] / [B, H, T]; the routing: gate [B, N, k] (moga_route),
+ * perm [B, T], inv [B, N, k], offsets [B, M+1] (moga_permute).  dO: the gradient with respect to the
+ * forward's output O, [B, H, N, D] with the shape's strides.
+ * Outputs: dQ, dK, dV [B, H, N, D] (same strides; a token routed to k groups receives the sum of
+ * its k contributions) and dgate [B, N, k] fp32 (the derivative with respect to each gate, summed
+ * over heads and channels: what the router's gate needs for its own backward).
+ * Kernels: one pass that scales and gathers dO and forms delta = <dO, o>, then two tensor-core
+ * launches (dQ; dK and dV) that recompute the softmax weights from lse, then the inverse
+ * permutation.  P, dS and the sorted-order gradients are rounded to bf16, accumulation is fp32.
+ * ws: moga_backward_workspace_bytes(s), 256-byte aligned; the device status word is at its start.
+ */
+size_t moga_backward_workspace_bytes(const moga_shape* s);
+moga_status moga_backward(const moga_shape* s, const void* Qp, const void* Kp, const void* Vp, const void* Op,
+                          const float* lse, const float* gate, const int32_t* perm, const int32_t* inv,
+                          const int32_t* offsets, const void* dO, void* dQ, void* dK, void* dV, float* dgate,
+                          void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Choice of the bf16 group-attention kernel (the paper has no counterpart: a tuning and test
  * switch).  Two kernels compute Eq. 1 inside the groups on the tensor cores.  The default
  * (MOGA_ATTN_AUTO, same as MOGA_ATTN_SINGLE) gives a block of 256 query rows to one SM.

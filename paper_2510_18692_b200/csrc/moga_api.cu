@@ -422,6 +422,62 @@ moga_status moga_visual_forward(const moga_shape* s, const void* X, const float*
   return launch_mean3(*s, w + v.A, w + v.Bs, lists->q_inv, w + v.C, O, cs);
 }
 
+namespace {
+struct BwdLayout {
+  size_t scratch, dOp, delta, dQp, dKp, dVp, total;
+};
+BwdLayout bwd_layout(const moga_shape& s) {
+  BwdLayout b{};
+  const size_t T = (size_t)s.N * s.k, row = elem_size(s.dtype) * (size_t)s.B * s.H * T * s.D;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = off;
+    off = align_up(off + bytes, kWsAlign);
+    return at;
+  };
+  b.scratch = take(ws_layout(s).scratch_end);
+  b.dOp = take(row);
+  b.delta = take(sizeof(float) * (size_t)s.B * s.H * T);
+  b.dQp = take(row);
+  b.dKp = take(row);
+  b.dVp = take(row);
+  b.total = off;
+  return b;
+}
+}  // namespace
+
+size_t moga_backward_workspace_bytes(const moga_shape* s) {
+  moga_status st;
+  if (!check_shape(s, &st)) return 0;
+  return bwd_layout(*s).total;
+}
+
+moga_status moga_backward(const moga_shape* s, const void* Qp, const void* Kp, const void* Vp, const void* Op,
+                          const float* lse, const float* gate, const int32_t* perm, const int32_t* inv,
+                          const int32_t* offsets, const void* dO, void* dQ, void* dK, void* dV, float* dgate,
+                          void* ws, size_t ws_bytes, void* stream) {
+  moga_status st;
+  if (!check_shape(s, &st)) return st;
+  if (s->dtype != MOGA_BF16 || s->D != 128) return MOGA_ERR_UNSUPPORTED;
+  if (s->N == 0) return MOGA_OK;
+  if (!PTR_OK(Qp) || !PTR_OK(Kp) || !PTR_OK(Vp) || !PTR_OK(Op) || !PTR_OK(lse) || !PTR_OK(gate) || !PTR_OK(perm) ||
+      !PTR_OK(inv) || !PTR_OK(offsets) || !PTR_OK(dO) || !PTR_OK(dQ) || !PTR_OK(dK) || !PTR_OK(dV) || !PTR_OK(dgate))
+    return MOGA_ERR_INVALID_ARG;
+  const BwdLayout b = bwd_layout(*s);
+  if (!check_ws(ws, ws_bytes, b.total, &st)) return st;
+  const WsLayout L = ws_layout(*s);
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  char* w = static_cast<char*>(ws);
+  if ((st = clear_header(w, L, cs)) != MOGA_OK) return st;
+  st = launch_attn_backward(*s, L, Qp, Kp, Vp, Op, lse, gate, perm, inv, offsets, dO, w + b.dOp,
+                            reinterpret_cast<float*>(w + b.delta), w + b.dQp, w + b.dKp, w + b.dVp, dgate, w, cs);
+  if (st != MOGA_OK) return st;
+  // back to token order: a token's gradient is the plain sum over its k assignments
+  if ((st = launch_unpermute(*s, w + b.dQp, inv, nullptr, dQ, cs)) != MOGA_OK) return st;
+  if ((st = launch_unpermute(*s, w + b.dKp, inv, nullptr, dK, cs)) != MOGA_OK) return st;
+  return launch_unpermute(*s, w + b.dVp, inv, nullptr, dV, cs);
+}
+
 moga_status moga_set_fused_topk(int32_t on) {
   set_fused_topk(on != 0);
   return MOGA_OK;

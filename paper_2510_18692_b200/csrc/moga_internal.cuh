@@ -116,6 +116,12 @@ moga_status launch_attn_bf16_scatter(const moga_shape& s, const WsLayout& L, con
 moga_status launch_attn_bf16_add(const moga_shape& s, const WsLayout& L, const void* Qp, const void* Kp,
                                  const void* Vp, const int32_t* offsets, const int32_t* asg, const float* gate,
                                  void* O, char* ws, cudaStream_t st);
+// Gradients of the bf16 group attention in sorted order (d_head = 128); see csrc/attn_bwd.cu.
+moga_status launch_attn_backward(const moga_shape& s, const WsLayout& L, const void* Qp, const void* Kp,
+                                 const void* Vp, const void* Op, const float* lse, const float* gate,
+                                 const int32_t* perm, const int32_t* inv, const int32_t* offsets, const void* dO,
+                                 void* dOp, float* delta, void* dQp, void* dKp, void* dVp, float* dgate, char* ws,
+                                 cudaStream_t st);
 void set_fused_topk(int on);
 bool fused_topk();
 

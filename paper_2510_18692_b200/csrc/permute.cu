@@ -153,7 +153,7 @@ unpermute_kernel(const uint4* __restrict__ Op, const int32_t* __restrict__ inv,
       for (int j = 0; j < KK; ++j) {
         const long long a = (long long)b * T + (long long)(n < N ? n : 0) * KK + j;
         pos[i][j] = __ldg(inv + a);
-        g[i][j] = __ldg(gate + a);
+        g[i][j] = gate != nullptr ? __ldg(gate + a) : 1.f;     // no gates: plain sum over the k assignments
       }
     }
 #pragma unroll
@@ -179,7 +179,7 @@ unpermute_kernel(const uint4* __restrict__ Op, const int32_t* __restrict__ inv,
       for (int j = 0; j < k; ++j) {
         const long long a = (long long)b * T + (long long)n * k + j;
         const int pos = __ldg(inv + a);
-        const float g = __ldg(gate + a);
+        const float g = gate != nullptr ? __ldg(gate + a) : 1.f;
         const uint4 raw = __ldg(Op + src_base + (long long)pos * vec_per_row + v);
         fma_vec(acc, raw, g, XT());
       }
