@@ -262,10 +262,11 @@ def main():
                          "attention, with one all-gather of the routing results as the only exchange (strong "
                          "scaling; the default for N > 1); 'layers' gives every rank its own layer (weak scaling, no "
                          "collective; the default for N = 1)")
-    ap.add_argument("--stage", default="all", choices=["all", "route", "visual"],
+    ap.add_argument("--stage", default="all", choices=["all", "route", "visual", "backward"],
                     help="'route' times moga_route alone on the config's X (a small resident set, for profiling); "
                          "'visual' times the whole visual-attention block: routed branch, the two static-group "
-                         "branches and their mean")
+                         "branches and their mean; 'backward' times moga_backward (gradients of the group attention and "
+                         "the gates) after a staged forward of the config")
     ap.add_argument("--attn-kernel", default="auto", choices=["auto", "single", "pair"],
                     help="bf16 group-attention kernel (moga_set_attn_kernel): the one-CTA kernel (default) or the "
                          "CTA-pair kernel, for A/B runs and profiles")
@@ -300,6 +301,8 @@ def main():
         return run_route_only(mb, cfg, dev, args)
     if args.stage == "visual":
         return run_visual_block(mb, cfg, dev, args)
+    if args.stage == "backward":
+        return run_backward(mb, cfg, dev, args)
     inp = make_inputs(cfg, device=dev)
     sh = mb.make_shape(cfg)
     ws = mb.alloc_workspace(mb.moga_workspace_bytes(sh), dev)
@@ -469,6 +472,61 @@ def run_route_only(mb, cfg, dev, args):
     print(json.dumps({"stage": "route", "config": config_dict(cfg), "ms": ms, "GB/s": by / ms / 1e6,
                       "frac_hbm": by / ms / 1e6 / peaks["hbm_gbs"], "peak_source": peaks["source"],
                       "device_status": mb.moga_last_device_status(ws)[0]}))
+    return 0
+
+
+def run_backward(mb, cfg, dev, args):
+    """moga_backward on the config's layer: a staged forward keeps the sorted-order tensors and lse, a
+    random upstream gradient is drawn, and the backward call is timed (bf16, d_head = 128)."""
+    inp = make_inputs(cfg, device=dev)
+    sh = mb.make_shape(cfg)
+    T = cfg.T
+    ws = mb.alloc_workspace(mb.moga_scratch_bytes(sh), dev)
+    gid = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.int32, device=dev)
+    gate = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.float32, device=dev)
+    perm = torch.empty(cfg.B, T, dtype=torch.int32, device=dev)
+    inv = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.int32, device=dev)
+    offsets = torch.empty(cfg.B, cfg.M + 1, dtype=torch.int32, device=dev)
+    Qp, Kp, Vp, Op = (torch.empty(cfg.B, cfg.H, T, cfg.D, dtype=inp["Q"].dtype, device=dev) for _ in range(4))
+    lse = torch.empty(cfg.B, cfg.H, T, dtype=torch.float32, device=dev)
+    mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], gid, gate, None, ws)
+    mb.moga_permute(sh, gid, inp["Q"], inp["K"], inp["V"], perm, inv, offsets, Qp, Kp, Vp, ws)
+    mb.moga_group_attn(sh, Qp, Kp, Vp, offsets, Op, lse, ws)
+    del inp["X"]
+    dO = torch.randn(inp["Q"].shape, device=dev, dtype=torch.float32).to(inp["Q"].dtype)
+    dQ, dK, dV = (torch.empty_like(inp["Q"]) for _ in range(3))
+    dgate = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.float32, device=dev)
+    wsb = mb.alloc_workspace(mb.moga_backward_workspace_bytes(sh), dev)
+
+    def step():
+        mb.moga_backward(sh, Qp, Kp, Vp, Op, lse, gate, perm, inv, offsets, dO, dQ, dK, dV, dgate, wsb)
+
+    for _ in range(args.warmup):
+        step()
+    code, detail = mb.moga_last_device_status(wsb)
+    if code != 0:
+        raise RuntimeError(f"device status {code} detail {detail:#x}")
+    clocks = ClockSampler(dev)
+    clocks.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    for e0, e1 in ev:
+        e0.record()
+        step()
+        e1.record()
+    torch.cuda.synchronize()
+    clk = clocks.stop()
+    ms = float(statistics.median(e0.elapsed_time(e1) for e0, e1 in ev))
+    sizes = np.diff(offsets.cpu().numpy(), axis=1)
+    fwd = sum(useful_flops(sizes[b], cfg.H, cfg.D) for b in range(cfg.B))
+    peaks = load_peaks()
+    print(json.dumps({
+        "stage": "backward", "config": config_dict(cfg), "ms": ms, "steps": args.steps,
+        "useful_tflop": 2.5 * fwd / 1e12, "executed_tflop": 3.5 * fwd / 1e12,
+        "useful_TFLOP/s": 2.5 * fwd / ms / 1e9, "executed_TFLOP/s": 3.5 * fwd / ms / 1e9,
+        "frac_tensor_sustained_executed": 3.5 * fwd / ms / 1e9 / peaks["bf16_tflops_sustained"],
+        "note": "useful = five GEMMs of 2 n^2 D per group (2.5 x the forward); executed = seven (the transposed "
+                "products are recomputed for dK / dV)", "clocks": clk}))
     return 0
 
 

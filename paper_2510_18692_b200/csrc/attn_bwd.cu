@@ -8,8 +8,8 @@
 // in sorted (group-major) order, do being the upstream gradient already multiplied by the gate.
 //
 // Two launches of one kernel template, both shaped like the forward kernel (TMA producer warp,
-// one MMA-issuing thread, four compute warps with one thread per TMEM lane, TMEM accumulators,
-// bounded waits), each work item one 128-row tile that stays resident while the other
+// one MMA-issuing thread, eight compute warps with two threads per TMEM lane (64 of the 128
+// columns each), TMEM accumulators, bounded waits), each work item one 128-row tile that stays resident while the other
 // operand's tiles stream past it:
 //   kModeQ   item = 128 query rows (Q, dO resident); streams the group's K / V tiles:
 //            T0 = Q K^T, T1 = dO V^T  ->  dS (bf16, over T1)  ->  dQ += dS K
@@ -21,7 +21,9 @@
 // operand of the accumulating MMAs: the same operand forms as the forward kernel, at the price of
 // seven GEMMs per tile pair instead of five.  The tensor pipe and the compute warps alternate
 // (one tile pair in flight); this kernel is the first correct form, not a tuned one.
-// TMEM: T0 [0,128) T1 [128,256) acc0 [256,384) acc1 [384,512).
+// TMEM: T0 [0,128) T1 [128,256) acc0 [256,384) acc1 [384,512); the bf16 results of the compute warps
+// overwrite columns [0,32) and [64,96) of the T region they were computed from (each half of the
+// threads writes inside the columns it has already read).
 #include "attn_common.cuh"
 
 namespace moga {
@@ -30,7 +32,7 @@ namespace {
 using namespace attn;
 using namespace sm100;
 
-constexpr int kThreads = 256;          // warp 0 producer, warp 1 MMA, warps 4-7 compute
+constexpr int kThreads = 384;          // warp 0 producer, warp 1 MMA, warps 4-11 compute (two per TMEM lane quarter)
 constexpr int kD = 128;
 constexpr int kTile = 128;
 constexpr int kBoxBytes = kTile * 128;           // 128 rows x 64 columns
@@ -38,8 +40,8 @@ constexpr int kTileBytes = 2 * kBoxBytes;        // 32 KB
 constexpr int NS = 2;                            // ring depth of the streamed tile pairs
 constexpr int kSmemR = 0;                        // resident pair
 constexpr int kSmemS = 2 * kTileBytes;           // streamed pairs
-constexpr int kSmemVec = kSmemS + NS * 2 * kTileBytes;   // 4 warps x (128 lse + 128 delta) floats
-constexpr int kSmemBar = kSmemVec + 4 * 256 * 4;
+constexpr int kSmemVec = kSmemS + NS * 2 * kTileBytes;   // 8 warps x (64 lse + 64 delta) floats
+constexpr int kSmemBar = kSmemVec + 8 * 128 * 4;
 constexpr int kNumBars = 2 + 2 * NS + 4;
 constexpr int kSmemTotal = kSmemBar + 8 * kNumBars + 16;
 constexpr int kDynSmem = kSmemTotal + 1024;
@@ -83,9 +85,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
       mbar_init(bar(S_EMPTY + i), 1);
     }
     mbar_init(bar(T_FULL), 1);
-    mbar_init(bar(E_FULL), kTile);
+    mbar_init(bar(E_FULL), 2 * kTile);
     mbar_init(bar(ACC_FULL), 1);
-    mbar_init(bar(ACC_EMPTY), kTile);
+    mbar_init(bar(ACC_EMPTY), 2 * kTile);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -151,13 +153,13 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
           mma_ss(tmem + t * kTile, ra + o, sb + o, hi, idesc_t, kk > 0);
         }
       };
-      // acc[a] (+)= E[e] S[t]   (E: bf16 over the first 64 columns of T[e])
+      // acc[a] (+)= E[e] S[t]   (E: bf16, streamed rows 0-63 in columns [0,32) of T[e], rows 64-127 in [64,96))
       auto issue_acc = [&](int a, int e, int t, uint32_t stage, bool accumulate) {
         const uint32_t vb = desc_lo(stage + t * kTileBytes, kBoxBytes);
 #pragma unroll
         for (int kk = 0; kk < kTile / 16; ++kk)
-          mma_ts(tmem + 256 + a * 128, tmem + e * kTile + kk * 8, vb + ((kk * 2048) >> 4), hi, idesc_a,
-                 (accumulate || kk > 0) ? 1u : 0u);
+          mma_ts(tmem + 256 + a * 128, tmem + e * kTile + (kk / 4) * 64 + (kk % 4) * 8, vb + ((kk * 2048) >> 4), hi,
+                 idesc_a, (accumulate || kk > 0) ? 1u : 0u);
       };
       uint32_t nit = 0, ns = 0, nt = 0;
       bool ok = true;
@@ -199,10 +201,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
   } else if (warp >= 4) {
     // ===================================================================== compute + epilogue
     const int q = warp & 3;
+    const int half = (warp - 4) >> 2;              // which 64 of the tile's 128 columns this thread handles
     const int r = q * 32 + lane;                   // row of the resident tile = TMEM lane
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
-    const uint32_t tT0 = tmem + lane_off, tT1 = tmem + lane_off + kTile;
-    float* wvec = reinterpret_cast<float*>(smem + kSmemVec) + q * 256;   // this warp's copy of the column vectors
+    const uint32_t tT0 = tmem + lane_off + half * 64, tT1 = tmem + lane_off + kTile + half * 64;
+    float* wvec = reinterpret_cast<float*>(smem + kSmemVec) + (warp - 4) * 128;   // this warp's column vectors
     const float log2e = 1.4426950408889634f;
     uint32_t nit = 0, nt = 0;
     bool ok = true;
@@ -224,11 +227,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
           // lse and delta of the streamed query rows, per column: each warp keeps its own copy
           __syncwarp();
 #pragma unroll
-          for (int m = 0; m < 4; ++m) {
-            const int c = lane + 32 * m;
-            const bool in = c < ncols;
-            wvec[c] = in ? args.lse[vbase + col0 + c] * log2e : 0.f;
-            wvec[128 + c] = in ? args.delta[vbase + col0 + c] : 0.f;
+          for (int m = 0; m < 2; ++m) {
+            const int c = lane + 32 * m, col = half * 64 + c;
+            const bool in = col < ncols;
+            wvec[c] = in ? args.lse[vbase + col0 + col] * log2e : 0.f;
+            wvec[64 + c] = in ? args.delta[vbase + col0 + col] : 0.f;
           }
           __syncwarp();
         }
@@ -236,7 +239,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {             // 32 columns at a time
+        for (int ch = 0; ch < 2; ++ch) {             // 32 of this thread's 64 columns at a time
           uint32_t t0[32], t1[32];
           tmem_ld32(tT0 + ch * 32, t0);
           tmem_ld32(tT1 + ch * 32, t1);
@@ -247,9 +250,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
             float pv[2], dv[2];
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
-              const int col = ch * 32 + c + e;
-              const float l2 = Mode == kModeQ ? row_lse : wvec[col];
-              const float dl = Mode == kModeQ ? row_delta : wvec[128 + col];
+              const int lc = ch * 32 + c + e, col = half * 64 + lc;
+              const float l2 = Mode == kModeQ ? row_lse : wvec[lc];
+              const float dl = Mode == kModeQ ? row_delta : wvec[64 + lc];
               float p = ex2(fmaf(__uint_as_float(t0[c + e]), scale_log2, -l2));
               p = col < ncols ? p : 0.f;             // columns past the group's end: no weight
               pv[e] = p;
@@ -260,7 +263,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
             ep[c >> 1] = *reinterpret_cast<uint32_t*>(&a);
             ed[c >> 1] = *reinterpret_cast<uint32_t*>(&b);
           }
-          // chunk ch of T0 / T1 has been read: its bf16 results may overwrite columns [16 ch, 16 ch + 16)
+          // chunk ch of this thread's columns has been read: its bf16 results overwrite the first
+          // 16 (ch) / next 16 columns of the same 64-column range
           if (Mode == kModeKV) tmem_st16(tT0 + ch * 16, ep);
           tmem_st16(tT1 + ch * 16, ed);
         }
@@ -277,7 +281,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
       for (int a = 0; a < (Mode == kModeKV ? 2 : 1); ++a) {
         __nv_bfloat16* out = (a == 0 ? args.out0 : args.out1) + (vbase + row) * kD;
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
+        for (int cc = 0; cc < 2; ++cc) {
+          const int ch = half * 2 + cc;            // this thread's half of the accumulator columns
           uint32_t acc[32];
           tmem_ld32(tmem + lane_off + 256 + a * 128 + ch * 32, acc);
           tmem_wait_ld();
