@@ -91,3 +91,32 @@ def test_backward_rejects_unsupported_shapes(mb):
     with pytest.raises(mb.MogaError) as e:
         mb.moga_backward(sh, t, t, t, t, t, t, t, t, t, t, t, t, t, t, ws)
     assert e.value.code == 2
+
+
+def test_backward_clip_size_one_head(mb):
+    """The single-clip workload (32,760 tokens, groups of ~4,100: 32 tiles per item, 64-bit offsets
+    in play for the other heads' rows): gradients of head 0 against the oracle run on that head
+    alone (heads are independent in dQ, dK, dV; dgate sums over heads and is checked in the small
+    cases)."""
+    from paper_2510_18692_b200.inputs import CONFIGS
+    cfg = CONFIGS["clip_bf16"]
+    inp = make_inputs(cfg, device="cuda")
+    sh, fw = _staged_forward(mb, cfg, inp)
+    g = torch.Generator(device="cuda").manual_seed(7)
+    dO = torch.randn(cfg.B, cfg.H, cfg.N, cfg.D, generator=g, device="cuda").to(torch.bfloat16)
+    dQ, dK, dV = (torch.empty_like(inp["Q"]) for _ in range(3))
+    dgate = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.float32, device="cuda")
+    ws = mb.alloc_workspace(mb.moga_backward_workspace_bytes(sh))
+    mb.moga_backward(sh, fw["Qp"], fw["Kp"], fw["Vp"], fw["Op"], fw["lse"], fw["gate"], fw["perm"], fw["inv"],
+                     fw["offsets"], dO, dQ, dK, dV, dgate, ws)
+    assert mb.moga_last_device_status(ws) == (0, 0)
+    h = 0
+    want = oracle.backward(to_np32(inp["Q"][:, h:h + 1]), to_np32(inp["K"][:, h:h + 1]), to_np32(inp["V"][:, h:h + 1]),
+                           fw["gid"].cpu().numpy(), fw["gate"].double().cpu().numpy(), to_np32(dO[:, h:h + 1]),
+                           cfg.scale, cfg.M)
+    for name, got, ref in (("dQ", dQ, want[0]), ("dK", dK, want[1]), ("dV", dV, want[2])):
+        got = got[:, h:h + 1].double().cpu().numpy()
+        err = np.abs(got - ref)
+        rel = float(np.sqrt((err ** 2).sum() / (ref ** 2).sum()))
+        print(f"{name}: rel fro {rel:.3e}  max err {err.max():.3e}  max |ref| {np.abs(ref).max():.3e}")
+        assert np.all(np.isfinite(got)) and rel <= 1e-2, (name, rel)
