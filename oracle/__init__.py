@@ -293,3 +293,41 @@ def backward(Q, K, V, gid, gate, dO, scale, M):
                 np.add.at(dV[b, h], tok, dv)
     return dQ, dK, dV, dgate
 
+
+def route_backward(X, Wr, bias, gid, dgate, gate_mode):
+    """Gradient of the router (Eq. 2-3 and the gate of Eq. 5) for a given dgate = dL/dgate.
+
+    The paper states no backward; this is the chain rule on its router: logits r = X W_r (+ bias),
+    the selected groups gid are fixed integers, and the gates are
+      mode ALL : gate_j = softmax(r)[g_j]                      -> dr_i = sum_j dgate_j p_{g_j} (delta(i, g_j) - p_i)
+      mode TOPK: gate_j = softmax over the k selected logits   -> dr_{g_i} = z_i (dgate_i - sum_j dgate_j z_j), 0 elsewhere
+    then dW_r = X^T dr, dbias = sum_n dr, dX = dr W_r^T.  All in fp64.
+    X [B,N,C], Wr [C,M], gid [B,N,k], dgate [B,N,k].  Returns dr [B,N,M], dX [B,N,C], dWr [C,M], dbias [M]."""
+    X = np.asarray(X, dtype=np.float64)
+    Wr = np.asarray(Wr, dtype=np.float64)
+    dgate = np.asarray(dgate, dtype=np.float64)
+    gid = np.asarray(gid)
+    B, N, C = X.shape
+    M = Wr.shape[1]
+    k = gid.shape[2]
+    r = X @ Wr + (0.0 if bias is None else np.asarray(bias, dtype=np.float64))
+    dr = np.zeros((B, N, M))
+    for b in range(B):
+        for n in range(N):
+            g = gid[b, n]
+            if gate_mode == GATE_SOFTMAX_ALL:
+                e = np.exp(r[b, n] - r[b, n].max())
+                p = e / e.sum()
+                for j in range(k):
+                    onehot = np.zeros(M)
+                    onehot[g[j]] = 1.0
+                    dr[b, n] += dgate[b, n, j] * p[g[j]] * (onehot - p)
+            else:
+                sel = r[b, n, g]
+                e = np.exp(sel - sel.max())
+                z = e / e.sum()
+                dr[b, n, g] = z * (dgate[b, n] - (dgate[b, n] * z).sum())
+    dX = dr @ Wr.T
+    dWr = np.einsum("bnc,bnm->cm", X, dr)
+    return dr, dX, dWr, dr.sum(axis=(0, 1))
+

@@ -467,3 +467,30 @@ def test_backward_oracle_special_cases():
     V2 = np.broadcast_to(V[:, :, :1], V.shape).copy()
     dQ2, dK2, dV2, _ = oracle.backward(Q, K, V2, gid2, gate, dO, 0.7, 1)
     assert np.abs(dQ2).max() < 1e-15 and np.abs(dK2).max() < 1e-15
+
+
+@pytest.mark.parametrize("gate_mode,k", [(GATE_SOFTMAX_ALL, 1), (GATE_SOFTMAX_ALL, 2), (GATE_SOFTMAX_TOPK, 2), (GATE_SOFTMAX_TOPK, 3)])
+def test_route_backward_oracle_against_autograd(gate_mode, k):
+    """The router's gradient against torch.autograd on the gate written with torch ops (softmax and
+    gather), with the oracle's own routing decision as the fixed index."""
+    rng = np.random.default_rng(5 + k)
+    B, N, C, M = 2, 23, 12, 6
+    X = rng.standard_normal((B, N, C)).astype(np.float32)
+    Wr = (rng.standard_normal((C, M)) / np.sqrt(C)).astype(np.float32)
+    bias = rng.standard_normal(M).astype(np.float32)
+    gid, gate, _ = oracle.route(X, Wr, bias, k, gate_mode)
+    dgate = rng.standard_normal((B, N, k))
+    dr, dX, dWr, dbias = oracle.route_backward(X, Wr, bias, gid, dgate, gate_mode)
+    tx, tw, tb = (torch.tensor(a.astype(np.float64), requires_grad=True) for a in (X, Wr, bias))
+    r = tx @ tw + tb
+    idx = torch.tensor(gid.astype(np.int64))
+    if gate_mode == GATE_SOFTMAX_ALL:
+        g = torch.softmax(r, -1).gather(-1, idx)
+    else:
+        g = torch.softmax(r.gather(-1, idx), -1)
+    assert np.abs(g.detach().numpy() - gate).max() < 1e-12          # the forward gate is the oracle's
+    gx, gw, gb = torch.autograd.grad(g, (tx, tw, tb), torch.tensor(dgate))
+    assert np.abs(dX - gx.numpy()).max() < 1e-12
+    assert np.abs(dWr - gw.numpy()).max() < 1e-12
+    assert np.abs(dbias - gb.numpy()).max() < 1e-12
+    assert np.abs(dr.sum(-1)).max() < 1e-12                          # softmax gradients sum to zero over the logits
