@@ -142,7 +142,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", self.index], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -158,6 +158,13 @@ class ClockSampler:
             out, _ = self.proc.communicate()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        if not out.strip():
+            # the timed region was shorter than the tool's start-up: one query right after it
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-i",
+                                      self.index], capture_output=True, text=True, timeout=10).stdout
+            except (OSError, subprocess.TimeoutExpired):
+                out = ""
         for line in out.strip().splitlines():
             f = [x.strip() for x in line.split(",")]
             if len(f) < 6:
@@ -489,10 +496,10 @@ def run_backward(mb, cfg, dev, args):
     offsets = torch.empty(cfg.B, cfg.M + 1, dtype=torch.int32, device=dev)
     Qp, Kp, Vp, Op = (torch.empty(cfg.B, cfg.H, T, cfg.D, dtype=inp["Q"].dtype, device=dev) for _ in range(4))
     lse = torch.empty(cfg.B, cfg.H, T, dtype=torch.float32, device=dev)
-    mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], gid, gate, None, ws)
+    logits = torch.empty(cfg.B, cfg.N, cfg.M, dtype=torch.float32, device=dev)
+    mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], gid, gate, logits, ws)
     mb.moga_permute(sh, gid, inp["Q"], inp["K"], inp["V"], perm, inv, offsets, Qp, Kp, Vp, ws)
     mb.moga_group_attn(sh, Qp, Kp, Vp, offsets, Op, lse, ws)
-    del inp["X"]
     dO = torch.randn(inp["Q"].shape, device=dev, dtype=torch.float32).to(inp["Q"].dtype)
     dQ, dK, dV = (torch.empty_like(inp["Q"]) for _ in range(3))
     dgate = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.float32, device=dev)
@@ -517,11 +524,29 @@ def run_backward(mb, cfg, dev, args):
     torch.cuda.synchronize()
     clk = clocks.stop()
     ms = float(statistics.median(e0.elapsed_time(e1) for e0, e1 in ev))
+    # the router's own backward from the dgate just computed
+    dX = torch.empty_like(inp["X"])
+    dWr = torch.empty_like(inp["Wr"])
+    dbias = torch.empty(cfg.M, dtype=torch.float32, device=dev)
+    wsr = mb.alloc_workspace(mb.moga_route_backward_workspace_bytes(sh), dev)
+    rb = []
+    for it in range(args.warmup + args.steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        mb.moga_route_backward(sh, inp["X"], inp["Wr"], logits, gid, dgate, dX, dWr, dbias, wsr)
+        e1.record()
+        torch.cuda.synchronize()
+        if it >= args.warmup:
+            rb.append(e0.elapsed_time(e1))
+    ms_route = float(statistics.median(rb))
     sizes = np.diff(offsets.cpu().numpy(), axis=1)
     fwd = sum(useful_flops(sizes[b], cfg.H, cfg.D) for b in range(cfg.B))
     peaks = load_peaks()
     print(json.dumps({
         "stage": "backward", "config": config_dict(cfg), "ms": ms, "steps": args.steps,
+        "route_backward_ms": ms_route,
+        "route_backward_GFLOP": 4.0 * cfg.B * cfg.N * cfg.C * cfg.M / 1e9,
+        "route_backward_TFLOP/s(fp32)": 4.0 * cfg.B * cfg.N * cfg.C * cfg.M / ms_route / 1e9,
         "useful_tflop": 2.5 * fwd / 1e12, "executed_tflop": 3.5 * fwd / 1e12,
         "useful_TFLOP/s": 2.5 * fwd / ms / 1e9, "executed_TFLOP/s": 3.5 * fwd / ms / 1e9,
         "frac_tensor_sustained_executed": 3.5 * fwd / ms / 1e9 / peaks["bf16_tflops_sustained"],

@@ -343,6 +343,21 @@ moga_status moga_backward(const moga_shape* s, const void* Qp, const void* Kp, c
                           void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Backward of the router (the paper states no backward pass: the chain rule on Eq. 2-3 and the
+ * gate of Eq. 5; the routing decision gid is a fixed integer choice).  Inputs: X [B, N, C] and W_r
+ * [C, M] as in moga_route, the logits [B, N, M] that moga_route wrote (its optional output), gid
+ * [B, N, k], and dgate [B, N, k] (from moga_backward); gate_mode as in the forward.
+ * Outputs: dWr [C, M] fp32, dbias [M] fp32 (nullable), dX [B, N, C] in the type of X (nullable: the
+ * gradient that reaches the token features through the router alone).  Deterministic: the sums over
+ * tokens are formed in a fixed order (per-slab partial sums, then a reduction), no atomics.
+ * fp32 ALUs throughout.  ws: moga_route_backward_workspace_bytes(s), 256-byte aligned.
+ */
+size_t moga_route_backward_workspace_bytes(const moga_shape* s);
+moga_status moga_route_backward(const moga_shape* s, const void* X, const float* Wr, const float* logits,
+                                const int32_t* gid, const float* dgate, void* dX, float* dWr, float* dbias, void* ws,
+                                size_t ws_bytes, void* stream);
+
+/*
  * Choice of the bf16 group-attention kernel (the paper has no counterpart: a tuning and test
  * switch).  Two kernels compute Eq. 1 inside the groups on the tensor cores.  The default
  * (MOGA_ATTN_AUTO, same as MOGA_ATTN_SINGLE) gives a block of 256 query rows to one SM.

@@ -22,7 +22,7 @@ EXPORTS = ("moga_workspace_bytes", "moga_scratch_bytes", "moga_status_string", "
            "moga_last_device_status", "moga_sort_static", "moga_balance_stats", "moga_stga_build", "moga_gather_rows",
            "moga_static_group_attn", "moga_mean3", "moga_forward_host_bytes", "moga_forward_host",
            "moga_visual_workspace_bytes", "moga_visual_forward", "moga_selftest_wait_timeout", "moga_set_attn_kernel", "moga_forward_routed", "moga_set_fused_topk", "moga_backward",
-           "moga_backward_workspace_bytes")
+           "moga_backward_workspace_bytes", "moga_route_backward", "moga_route_backward_workspace_bytes")
 
 MOGA_F32, MOGA_BF16 = 0, 1
 MOGA_ROUTE_AUTO, MOGA_ROUTE_ALU = 0, 1
@@ -59,7 +59,7 @@ lib = ctypes.CDLL(LIB_PATH)
 for _n in EXPORTS:
     getattr(lib, _n).restype = ctypes.c_int
 for _n in ("moga_workspace_bytes", "moga_scratch_bytes", "moga_static_scratch_bytes", "moga_forward_host_bytes",
-           "moga_visual_workspace_bytes", "moga_backward_workspace_bytes"):
+           "moga_visual_workspace_bytes", "moga_backward_workspace_bytes", "moga_route_backward", "moga_route_backward_workspace_bytes"):
     getattr(lib, _n).restype = ctypes.c_size_t
 lib.moga_status_string.restype = ctypes.c_char_p
 
@@ -190,6 +190,16 @@ def moga_forward_routed(shape, gid, gate, Q, K, V, O, ws, perm_out=None, offsets
     _check(lib.moga_forward_routed(ctypes.byref(shape), _ptr(gid), _ptr(gate), _ptr(Q), _ptr(K), _ptr(V), _ptr(O),
                                    _ptr(perm_out), _ptr(offsets_out), _ptr(ws), ctypes.c_size_t(ws.numel()),
                                    _stream()), "moga_forward_routed")
+
+
+def moga_route_backward_workspace_bytes(shape) -> int:
+    return int(lib.moga_route_backward_workspace_bytes(ctypes.byref(shape)))
+
+
+def moga_route_backward(shape, X, Wr, logits, gid, dgate, dX, dWr, dbias, ws):
+    _check(lib.moga_route_backward(ctypes.byref(shape), _ptr(X), _ptr(Wr), _ptr(logits), _ptr(gid), _ptr(dgate),
+                                   _ptr(dX), _ptr(dWr), _ptr(dbias), _ptr(ws), ctypes.c_size_t(ws.numel()),
+                                   _stream()), "moga_route_backward")
 
 
 def moga_backward_workspace_bytes(shape) -> int:

@@ -478,6 +478,26 @@ moga_status moga_backward(const moga_shape* s, const void* Qp, const void* Kp, c
   return launch_unpermute(*s, w + b.dVp, inv, nullptr, dV, cs);
 }
 
+size_t moga_route_backward_workspace_bytes(const moga_shape* s) {
+  moga_status st;
+  if (!check_shape(s, &st)) return 0;
+  return route_backward_bytes(*s);
+}
+
+moga_status moga_route_backward(const moga_shape* s, const void* X, const float* Wr, const float* logits,
+                                const int32_t* gid, const float* dgate, void* dX, float* dWr, float* dbias, void* ws,
+                                size_t ws_bytes, void* stream) {
+  moga_status st;
+  if (!check_shape(s, &st)) return st;
+  if (!PTR_OK(Wr) || !PTR_OK(dWr) || (dbias != nullptr && (reinterpret_cast<uintptr_t>(dbias) & 3u)) ||
+      (dX != nullptr && !aligned16(dX)))
+    return MOGA_ERR_INVALID_ARG;
+  if (s->N > 0 && (!PTR_OK(X) || !PTR_OK(logits) || !PTR_OK(gid) || !PTR_OK(dgate))) return MOGA_ERR_INVALID_ARG;
+  if (!check_ws(ws, ws_bytes, route_backward_bytes(*s), &st)) return st;
+  return launch_route_backward(*s, X, Wr, logits, gid, dgate, dX, dWr, dbias, static_cast<char*>(ws),
+                               static_cast<cudaStream_t>(stream));
+}
+
 moga_status moga_set_fused_topk(int32_t on) {
   set_fused_topk(on != 0);
   return MOGA_OK;

@@ -122,6 +122,11 @@ moga_status launch_attn_backward(const moga_shape& s, const WsLayout& L, const v
                                  const int32_t* perm, const int32_t* inv, const int32_t* offsets, const void* dO,
                                  void* dOp, float* delta, void* dQp, void* dKp, void* dVp, float* dgate, char* ws,
                                  cudaStream_t st);
+// Router backward (csrc/route_bwd.cu): scratch bytes and the launches.
+size_t route_backward_bytes(const moga_shape& s);
+moga_status launch_route_backward(const moga_shape& s, const void* X, const float* Wr, const float* logits,
+                                  const int32_t* gid, const float* dgate, void* dX, float* dWr, float* dbias, char* ws,
+                                  cudaStream_t st);
 void set_fused_topk(int on);
 bool fused_topk();
 

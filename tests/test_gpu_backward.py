@@ -120,3 +120,48 @@ def test_backward_clip_size_one_head(mb):
         rel = float(np.sqrt((err ** 2).sum() / (ref ** 2).sum()))
         print(f"{name}: rel fro {rel:.3e}  max err {err.max():.3e}  max |ref| {np.abs(ref).max():.3e}")
         assert np.all(np.isfinite(got)) and rel <= 1e-2, (name, rel)
+
+
+ROUTE_BWD = [
+    MogaConfig("rb_all_top1", 2, 1, 1500, 256, 64, 8, 1, "bf16", GATE_SOFTMAX_ALL, 61),
+    MogaConfig("rb_all_top2", 1, 1, 777, 136, 64, 5, 2, "bf16", GATE_SOFTMAX_ALL, 62),
+    MogaConfig("rb_topk", 1, 1, 3000, 320, 64, 64, 2, "bf16", GATE_SOFTMAX_TOPK, 63, zipf_bias=2.0),
+    MogaConfig("rb_f32", 1, 1, 1000, 96, 64, 16, 3, "f32", GATE_SOFTMAX_TOPK, 64),
+    MogaConfig("rb_m1", 1, 1, 300, 64, 64, 1, 1, "bf16", GATE_SOFTMAX_ALL, 65),
+]
+
+
+@pytest.mark.parametrize("cfg", ROUTE_BWD, ids=lambda c: c.name)
+def test_route_backward_matches_oracle(mb, cfg):
+    """dX, dW_r, dbias of the router against the fp64 oracle, from the GPU's own routing and logits.
+    Tolerances: dW_r and dbias are fp32 sums over the tokens (relative 1e-4 of the largest entry);
+    dX is rounded to the type of X (bf16: 2^-8 of the row's magnitude); dr itself depends on the
+    fp32 logits (2e-5) through a softmax."""
+    inp = make_inputs(cfg, device="cuda", heads=[])
+    sh = mb.make_shape(cfg)
+    ws = mb.alloc_workspace(mb.moga_scratch_bytes(sh))
+    gid = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.int32, device="cuda")
+    gate = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.float32, device="cuda")
+    logits = torch.empty(cfg.B, cfg.N, cfg.M, dtype=torch.float32, device="cuda")
+    mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], gid, gate, logits, ws)
+    g = torch.Generator(device="cuda").manual_seed(cfg.seed)
+    dgate = torch.randn(cfg.B, cfg.N, cfg.k, generator=g, device="cuda")
+    dX = torch.full_like(inp["X"], float("nan"))
+    dWr = torch.full_like(inp["Wr"], float("nan"))
+    dbias = torch.full((cfg.M,), float("nan"), device="cuda")
+    wsb = mb.alloc_workspace(mb.moga_route_backward_workspace_bytes(sh))
+    outs = []
+    for _ in range(2):
+        mb.moga_route_backward(sh, inp["X"], inp["Wr"], logits, gid, dgate, dX, dWr, dbias, wsb)
+        torch.cuda.synchronize()
+        outs.append((dX.clone(), dWr.clone(), dbias.clone()))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)                                   # fixed summation order: bit-reproducible
+    _, o_dX, o_dWr, o_db = oracle.route_backward(to_np32(inp["X"]), inp["Wr"].cpu().numpy(),
+                                                 None if inp["bias"] is None else inp["bias"].cpu().numpy(),
+                                                 gid.cpu().numpy(), dgate.double().cpu().numpy(), cfg.gate_mode)
+    got_w, got_b, got_x = dWr.double().cpu().numpy(), dbias.double().cpu().numpy(), dX.double().cpu().numpy()
+    assert np.abs(got_w - o_dWr).max() <= 1e-4 * max(np.abs(o_dWr).max(), 1e-6) + 1e-7
+    assert np.abs(got_b - o_db).max() <= 1e-4 * max(np.abs(o_db).max(), 1e-6) + 1e-6
+    tol = (2.0 ** -8 if cfg.dtype == "bf16" else 1e-5) * np.abs(o_dX).max(axis=-1, keepdims=True) + 1e-6
+    assert np.all(np.abs(got_x - o_dX) <= tol)
