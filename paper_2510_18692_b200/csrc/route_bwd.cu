@@ -112,75 +112,99 @@ route_dlogits_kernel(const float* __restrict__ logits, const int32_t* __restrict
   }
 }
 
-// dX[t, c] = sum_i dr[t, i] W[c, i].  Block: 32 tokens x 128 channels per pass; thread (tx, ty) of
-// 16 x 16 owns tokens ty*2, ty*2 + 1 and channels tx + 16 u, u < 8.
-constexpr int kDxTok = 32, kDxCh = 128;
+// Loads of four consecutive channels of X as fp32.
+__device__ __forceinline__ void load4(const float* p, float (&v)[4]) {
+  const float4 t = *reinterpret_cast<const float4*>(p);
+  v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+}
+__device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&v)[4]) {
+  const uint2 t = *reinterpret_cast<const uint2*>(p);
+  v[0] = __uint_as_float(t.x << 16); v[1] = __uint_as_float(t.x & 0xffff0000u);
+  v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xffff0000u);
+}
+__device__ __forceinline__ void store4(float* p, const float (&v)[4]) {
+  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+}
+__device__ __forceinline__ void store4(__nv_bfloat16* p, const float (&v)[4]) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+  *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+}
+
+// dX[t, c] = sum_i dr[t, i] W[c, i].  Block: 64 tokens, all channels in chunks of 128.  Thread
+// (lane = channel quad, warp = token octet) owns 8 tokens x 4 channels; per logit column it reads
+// two 16-byte words of dr (the same for the whole warp) and one of W, for 32 multiply-adds.
+// Dynamic shared memory: drT [M][64] and wT [M][128] floats.
+constexpr int kDxTok = 64, kDxCh = 128;
 template <typename XT>
 __global__ void __launch_bounds__(256)
 route_dx_kernel(const float* __restrict__ dr, const float* __restrict__ Wr, XT* __restrict__ dX, long long tokens, int C,
                 int M) {
-  __shared__ float sdr[kDxTok][kMaxM + 1];
-  __shared__ float sw[kDxCh][kMaxM + 1];
+  extern __shared__ __align__(16) float dx_smem[];
+  float* drT = dx_smem;                   // [M][kDxTok]
+  float* wT = dx_smem + M * kDxTok;       // [M][kDxCh]
   const long long t0 = (long long)blockIdx.x * kDxTok;
-  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int idx = threadIdx.x; idx < kDxTok * M; idx += 256) {
-    const int tt = idx / M, i = idx % M;
-    sdr[tt][i] = t0 + tt < tokens ? dr[(t0 + tt) * M + i] : 0.f;
+    const int i = idx / kDxTok, tt = idx % kDxTok;        // consecutive threads: consecutive tokens (no bank conflicts)
+    drT[i * kDxTok + tt] = t0 + tt < tokens ? dr[(t0 + tt) * M + i] : 0.f;
   }
   for (int c0 = 0; c0 < C; c0 += kDxCh) {
     __syncthreads();
     for (int idx = threadIdx.x; idx < kDxCh * M; idx += 256) {
-      const int cc = idx / M, i = idx % M;
-      sw[cc][i] = c0 + cc < C ? Wr[(size_t)(c0 + cc) * M + i] : 0.f;
+      const int i = idx / kDxCh, cc = idx % kDxCh;        // consecutive threads: consecutive channels
+      wT[i * kDxCh + cc] = c0 + cc < C ? Wr[(size_t)(c0 + cc) * M + i] : 0.f;
     }
     __syncthreads();
-    float acc[2][8];
+    float acc[8][4];
 #pragma unroll
-    for (int a = 0; a < 2; ++a)
+    for (int a = 0; a < 8; ++a)
 #pragma unroll
-      for (int u = 0; u < 8; ++u) acc[a][u] = 0.f;
+      for (int u = 0; u < 4; ++u) acc[a][u] = 0.f;
     for (int i = 0; i < M; ++i) {
-      float d[2];
+      const float4 d0 = *reinterpret_cast<const float4*>(drT + i * kDxTok + warp * 8);
+      const float4 d1 = *reinterpret_cast<const float4*>(drT + i * kDxTok + warp * 8 + 4);
+      const float4 w4 = *reinterpret_cast<const float4*>(wT + i * kDxCh + lane * 4);
+      const float d[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+      const float w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
-      for (int a = 0; a < 2; ++a) d[a] = sdr[ty * 2 + a][i];
+      for (int a = 0; a < 8; ++a)
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const float wv = sw[tx + 16 * u][i];
-#pragma unroll
-        for (int a = 0; a < 2; ++a) acc[a][u] = fmaf(d[a], wv, acc[a][u]);
-      }
+        for (int u = 0; u < 4; ++u) acc[a][u] = fmaf(d[a], w[u], acc[a][u]);
     }
+    const int c = c0 + lane * 4;
+    if (c < C) {
 #pragma unroll
-    for (int a = 0; a < 2; ++a) {
-      const long long t = t0 + ty * 2 + a;
-      if (t < tokens) {
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int c = c0 + tx + 16 * u;
-          if (c < C) dX[t * C + c] = from_f32<XT>(acc[a][u]);
-        }
+      for (int a = 0; a < 8; ++a) {
+        const long long t = t0 + warp * 8 + a;
+        if (t < tokens) store4(dX + t * C + c, acc[a]);
       }
     }
   }
 }
 
 // part[slab, c, i] = sum over the slab's tokens of X[t, c] dr[t, i], for the block's 128 channels.
-// Thread: channel c = c0 + (threadIdx.x & 127), and half of the M columns (threadIdx.x >> 7).
+// Thread (lane = channel quad, warp = group of MC = ceil(M / 8) logit columns) owns 4 channels x MC
+// columns; per token it reads 4 channels of X and MC values of dr (the same for the whole warp).
+// (First form: the X loads, eight bytes per thread and token with four in flight, are latency-bound;
+// measured 10-15 TFLOP/s fp32 at the minute-long size (25-39 ms, 3-5 % of the backward step).  Wider column blocks per thread were tried and
+// were slower at one block per SM; staging X through shared memory with cp.async is the next step.)
 template <typename XT>
 __global__ void __launch_bounds__(256)
 route_dw_partial_kernel(const XT* __restrict__ X, const float* __restrict__ dr, float* __restrict__ part,
                         long long tokens, int C, int M) {
-  constexpr int kTokTile = 32;
-  __shared__ float sdr[kTokTile][kMaxM];
+  constexpr int kTokTile = 64;
+  __shared__ __align__(16) float sdr[kTokTile][kMaxM];
   const int slab = blockIdx.y;
-  const int c = blockIdx.x * kWcChunk + (threadIdx.x & (kWcChunk - 1));
-  const int half = threadIdx.x >> 7;
-  const int mh = (M + 1) / 2, i0 = half * mh, i1 = min(M, i0 + mh);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int c = blockIdx.x * kWcChunk + lane * 4;
+  const int MC = (M + 7) / 8, i0 = warp * MC;
   const long long per = (tokens + kSlabs - 1) / kSlabs;
   const long long ta = (long long)slab * per, tb = min(tokens, ta + per);
-  float acc[kMaxM / 2];
+  float acc[4][kMaxM / 8];
 #pragma unroll
-  for (int i = 0; i < kMaxM / 2; ++i) acc[i] = 0.f;
+  for (int u = 0; u < 4; ++u)
+#pragma unroll
+    for (int i = 0; i < kMaxM / 8; ++i) acc[u][i] = 0.f;
   for (long long t0 = ta; t0 < tb; t0 += kTokTile) {
     __syncthreads();
     for (int idx = threadIdx.x; idx < kTokTile * M; idx += 256) {
@@ -188,21 +212,29 @@ route_dw_partial_kernel(const XT* __restrict__ X, const float* __restrict__ dr, 
       sdr[tt][i] = t0 + tt < tb ? dr[(t0 + tt) * M + i] : 0.f;
     }
     __syncthreads();
-    if (c < C) {
+    if (c < C && i0 < M) {
+      const int nt = (int)min((long long)kTokTile, tb - t0);
 #pragma unroll 4
-      for (int tt = 0; tt < kTokTile; ++tt) {
-        if (t0 + tt >= tb) break;
-        const float x = to_f32<XT>(X[(t0 + tt) * C + c]);
+      for (int tt = 0; tt < nt; ++tt) {
+        float x[4];
+        load4(X + (t0 + tt) * C + c, x);
 #pragma unroll
-        for (int i = 0; i < kMaxM / 2; ++i)
-          if (i0 + i < i1) acc[i] = fmaf(x, sdr[tt][i0 + i], acc[i]);
+        for (int i = 0; i < kMaxM / 8; ++i) {
+          if (i < MC) {
+            const float dv = i0 + i < M ? sdr[tt][i0 + i] : 0.f;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) acc[u][i] = fmaf(x[u], dv, acc[u][i]);
+          }
+        }
       }
     }
   }
   if (c < C)
 #pragma unroll
-    for (int i = 0; i < kMaxM / 2; ++i)
-      if (i0 + i < i1) part[((size_t)slab * C + c) * M + i0 + i] = acc[i];
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int i = 0; i < kMaxM / 8; ++i)
+        if (i < MC && i0 + i < M) part[((size_t)slab * C + c + u) * M + i0 + i] = acc[u][i];
 }
 
 // dWr[c, i] = sum over slabs (in order) of part[slab, c, i];  dbias[i] = sum over blocks of colsum
@@ -247,16 +279,23 @@ moga_status launch_route_backward(const moga_shape& s, const void* X, const floa
   route_dlogits_kernel<<<nblk, kDrThreads, 0, st>>>(logits, gid, dgate, dr, colsum, tokens, s.M, s.k, s.gate_mode);
   MOGA_CUDA_OK(cudaGetLastError());
   dim3 wgrid((s.C + kWcChunk - 1) / kWcChunk, kSlabs);
+  const size_t dx_smem_bytes = sizeof(float) * (size_t)s.M * (kDxTok + kDxCh);
   if (s.dtype == MOGA_BF16) {
-    if (dX)
-      route_dx_kernel<__nv_bfloat16><<<(unsigned)((tokens + kDxTok - 1) / kDxTok), 256, 0, st>>>(
+    if (dX) {
+      MOGA_CUDA_OK(cudaFuncSetAttribute(route_dx_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)(sizeof(float) * kMaxM * (kDxTok + kDxCh))));
+      route_dx_kernel<__nv_bfloat16><<<(unsigned)((tokens + kDxTok - 1) / kDxTok), 256, dx_smem_bytes, st>>>(
           dr, Wr, static_cast<__nv_bfloat16*>(dX), tokens, s.C, s.M);
+    }
     route_dw_partial_kernel<__nv_bfloat16><<<wgrid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(X), dr, part,
                                                                   tokens, s.C, s.M);
   } else {
-    if (dX)
-      route_dx_kernel<float><<<(unsigned)((tokens + kDxTok - 1) / kDxTok), 256, 0, st>>>(
+    if (dX) {
+      MOGA_CUDA_OK(cudaFuncSetAttribute(route_dx_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)(sizeof(float) * kMaxM * (kDxTok + kDxCh))));
+      route_dx_kernel<float><<<(unsigned)((tokens + kDxTok - 1) / kDxTok), 256, dx_smem_bytes, st>>>(
           dr, Wr, static_cast<float*>(dX), tokens, s.C, s.M);
+    }
     route_dw_partial_kernel<float><<<wgrid, 256, 0, st>>>(static_cast<const float*>(X), dr, part, tokens, s.C, s.M);
   }
   MOGA_CUDA_OK(cudaGetLastError());
