@@ -2,7 +2,7 @@
 oracle: the forward is run with the stage calls (which keep the sorted-order tensors and lse the
 backward needs), an upstream gradient dO is drawn, and dQ, dK, dV, dgate are compared.
 
-Tolerance (derived in the design doc): the kernels round the softmax weights, dS, the scaled upstream
+Tolerance: the kernels round the softmax weights, dS, the scaled upstream
 gradient and the sorted-order results to bf16 (2^-9 each) and accumulate in fp32, and the forward
 output they take as saved input is itself bf16: relative Frobenius error <= 1e-2 per gradient
 (measured ~3e-3), largest error <= 2^-5 of the tensor's largest magnitude."""
