@@ -24,6 +24,8 @@
 // TMEM: T0 [0,128) T1 [128,256) acc0 [256,384) acc1 [384,512); the bf16 results of the compute warps
 // overwrite columns [0,32) and [64,96) of the T region they were computed from (each half of the
 // threads writes inside the columns it has already read).
+#include <type_traits>
+
 #include "attn_common.cuh"
 
 namespace moga {
@@ -215,10 +217,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
       const int row = it.row0 + r;
       const bool live = row < it.qhi;
       const size_t vbase = (size_t)it.bh * T;
-      float row_lse = 0.f, row_delta = 0.f;
+      float row_lse = 0.f, row_delta = 0.f;       // minus lse * log2e and minus delta * scale of this row
       if (Mode == kModeQ && live) {
-        row_lse = args.lse[vbase + row] * log2e;
-        row_delta = args.delta[vbase + row];
+        row_lse = -args.lse[vbase + row] * log2e;
+        row_delta = -args.delta[vbase + row] * scale;
       }
       for (int j = 0; j < ntiles && ok; ++j, ++nt) {
         const int col0 = it.klo + j * kTile;
@@ -230,16 +232,18 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
           for (int m = 0; m < 2; ++m) {
             const int c = lane + 32 * m, col = half * 64 + c;
             const bool in = col < ncols;
-            wvec[c] = in ? args.lse[vbase + col0 + col] * log2e : 0.f;
-            wvec[64 + c] = in ? args.delta[vbase + col0 + col] : 0.f;
+            wvec[c] = in ? -args.lse[vbase + col0 + col] * log2e : 0.f;
+            wvec[64 + c] = in ? -args.delta[vbase + col0 + col] * scale : 0.f;
           }
           __syncwarp();
         }
         ok = __all_sync(0xffffffffu, wait(T_FULL, nt & 1u, 7));
         if (!ok) break;
         tc_fence_after();
-#pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {             // 32 of this thread's 64 columns at a time
+        // p = 2^(t0 * scale_log2 - lse * log2e),  ds = p * (t1 * scale - delta * scale): packed fp32 pairs.
+        // A tile that reaches past the group's end takes the variant that zeroes those columns' p.
+        const float2 sl2 = make_float2(scale_log2, scale_log2), sc2 = make_float2(scale, scale);
+        auto chunk = [&](int ch, auto masked) {
           uint32_t t0[32], t1[32];
           tmem_ld32(tT0 + ch * 32, t0);
           tmem_ld32(tT1 + ch * 32, t1);
@@ -247,26 +251,40 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
           uint32_t ep[16], ed[16];
 #pragma unroll
           for (int c = 0; c < 32; c += 2) {
-            float pv[2], dv[2];
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-              const int lc = ch * 32 + c + e, col = half * 64 + lc;
-              const float l2 = Mode == kModeQ ? row_lse : wvec[lc];
-              const float dl = Mode == kModeQ ? row_delta : wvec[64 + lc];
-              float p = ex2(fmaf(__uint_as_float(t0[c + e]), scale_log2, -l2));
-              p = col < ncols ? p : 0.f;             // columns past the group's end: no weight
-              pv[e] = p;
-              dv[e] = p * (__uint_as_float(t1[c + e]) - dl) * scale;
+            const int lc = ch * 32 + c;
+            float2 nl2, nds;                          // minus lse * log2e, minus delta * scale, of the two columns
+            if (Mode == kModeQ) {
+              nl2 = make_float2(row_lse, row_lse);
+              nds = make_float2(row_delta, row_delta);
+            } else {
+              nl2 = *reinterpret_cast<const float2*>(wvec + lc);
+              nds = *reinterpret_cast<const float2*>(wvec + 64 + lc);
             }
-            __nv_bfloat162 a = __floats2bfloat162_rn(pv[0], pv[1]);
-            __nv_bfloat162 b = __floats2bfloat162_rn(dv[0], dv[1]);
+            const float2 x = __ffma2_rn(make_float2(__uint_as_float(t0[c]), __uint_as_float(t0[c + 1])), sl2, nl2);
+            float2 pe = make_float2(ex2(x.x), ex2(x.y));
+            if (decltype(masked)::value) {
+              const int col = half * 64 + lc;
+              pe.x = col < ncols ? pe.x : 0.f;
+              pe.y = col + 1 < ncols ? pe.y : 0.f;
+            }
+            const float2 u = __ffma2_rn(make_float2(__uint_as_float(t1[c]), __uint_as_float(t1[c + 1])), sc2, nds);
+            const float2 ds = __fmul2_rn(pe, u);
+            __nv_bfloat162 a = __floats2bfloat162_rn(pe.x, pe.y);
+            __nv_bfloat162 b = __floats2bfloat162_rn(ds.x, ds.y);
             ep[c >> 1] = *reinterpret_cast<uint32_t*>(&a);
             ed[c >> 1] = *reinterpret_cast<uint32_t*>(&b);
           }
           // chunk ch of this thread's columns has been read: its bf16 results overwrite the first
-          // 16 (ch) / next 16 columns of the same 64-column range
+          // 16 (ch = 0) / next 16 columns of the same 64-column range
           if (Mode == kModeKV) tmem_st16(tT0 + ch * 16, ep);
           tmem_st16(tT1 + ch * 16, ed);
+        };
+        if (ncols < kTile) {
+          chunk(0, std::true_type{});
+          chunk(1, std::true_type{});
+        } else {
+          chunk(0, std::false_type{});
+          chunk(1, std::false_type{});
         }
         tmem_wait_st();
         tc_fence_before();
