@@ -323,7 +323,8 @@ moga_status moga_last_device_status(void* ws, void* stream, uint32_t* detail);
 /*
  * Backward of the routed group attention (the paper states no backward pass: this is the chain
  * rule applied to Eq. 1 inside each group and the gate of Eq. 5; the routing decision carries no
- * gradient).  bf16, d_head = 128 (else MOGA_ERR_UNSUPPORTED).
+ * gradient).  bf16 with d_head = 128 and fp32 with d_head 64 or 128; bf16 with d_head = 64 returns
+ * MOGA_ERR_UNSUPPORTED.
  * Saved from a forward made of the stage calls, all in sorted order: Qp, Kp, Vp (moga_permute),
  * Op and lse (moga_group_attn), [B, H, T, D] / [B, H, T]; the routing: gate [B, N, k] (moga_route),
  * perm [B, T], inv [B, N, k], offsets [B, M+1] (moga_permute).  dO: the gradient with respect to the
@@ -334,6 +335,7 @@ moga_status moga_last_device_status(void* ws, void* stream, uint32_t* detail);
  * Kernels: one pass that scales and gathers dO and forms delta = <dO, o>, then two tensor-core
  * launches (dQ; dK and dV) that recompute the softmax weights from lse, then the inverse
  * permutation.  P, dS and the sorted-order gradients are rounded to bf16, accumulation is fp32.
+ * fp32 tensors take the same three steps on the fp32 ALUs, nothing rounded below fp32.
  * ws: moga_backward_workspace_bytes(s), 256-byte aligned; the device status word is at its start.
  */
 size_t moga_backward_workspace_bytes(const moga_shape* s);

@@ -458,7 +458,7 @@ moga_status moga_backward(const moga_shape* s, const void* Qp, const void* Kp, c
                           void* ws, size_t ws_bytes, void* stream) {
   moga_status st;
   if (!check_shape(s, &st)) return st;
-  if (s->dtype != MOGA_BF16 || s->D != 128) return MOGA_ERR_UNSUPPORTED;
+  if (s->dtype == MOGA_BF16 && s->D != 128) return MOGA_ERR_UNSUPPORTED;
   if (s->N == 0) return MOGA_OK;
   if (!PTR_OK(Qp) || !PTR_OK(Kp) || !PTR_OK(Vp) || !PTR_OK(Op) || !PTR_OK(lse) || !PTR_OK(gate) || !PTR_OK(perm) ||
       !PTR_OK(inv) || !PTR_OK(offsets) || !PTR_OK(dO) || !PTR_OK(dQ) || !PTR_OK(dK) || !PTR_OK(dV) || !PTR_OK(dgate))
@@ -469,8 +469,15 @@ moga_status moga_backward(const moga_shape* s, const void* Qp, const void* Kp, c
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   char* w = static_cast<char*>(ws);
   if ((st = clear_header(w, L, cs)) != MOGA_OK) return st;
-  st = launch_attn_backward(*s, L, Qp, Kp, Vp, Op, lse, gate, perm, inv, offsets, dO, w + b.dOp,
-                            reinterpret_cast<float*>(w + b.delta), w + b.dQp, w + b.dKp, w + b.dVp, dgate, w, cs);
+  if (s->dtype == MOGA_BF16) {
+    st = launch_attn_backward(*s, L, Qp, Kp, Vp, Op, lse, gate, perm, inv, offsets, dO, w + b.dOp,
+                              reinterpret_cast<float*>(w + b.delta), w + b.dQp, w + b.dKp, w + b.dVp, dgate, w, cs);
+  } else {
+    auto f = [](const void* x) { return static_cast<const float*>(x); };
+    auto g = [&](size_t at) { return reinterpret_cast<float*>(w + at); };
+    st = launch_attn_backward_f32(*s, f(Qp), f(Kp), f(Vp), f(Op), lse, gate, perm, inv, offsets, f(dO), g(b.dOp),
+                                  g(b.delta), g(b.dQp), g(b.dKp), g(b.dVp), dgate, cs);
+  }
   if (st != MOGA_OK) return st;
   // back to token order: a token's gradient is the plain sum over its k assignments
   if ((st = launch_unpermute(*s, w + b.dQp, inv, nullptr, dQ, cs)) != MOGA_OK) return st;

@@ -122,6 +122,12 @@ moga_status launch_attn_backward(const moga_shape& s, const WsLayout& L, const v
                                  const int32_t* perm, const int32_t* inv, const int32_t* offsets, const void* dO,
                                  void* dOp, float* delta, void* dQp, void* dKp, void* dVp, float* dgate, char* ws,
                                  cudaStream_t st);
+// The same gradients for fp32 tensors on the fp32 ALUs (d_head 64 or 128); see csrc/attn_bwd_f32.cu.
+moga_status launch_attn_backward_f32(const moga_shape& s, const float* Qp, const float* Kp, const float* Vp,
+                                     const float* Op, const float* lse, const float* gate, const int32_t* perm,
+                                     const int32_t* inv, const int32_t* offsets, const float* dO, float* dOp,
+                                     float* delta, float* dQp, float* dKp, float* dVp, float* dgate,
+                                     cudaStream_t st);
 // Router backward (csrc/route_bwd.cu): scratch bytes and the launches.
 size_t route_backward_bytes(const moga_shape& s);
 moga_status launch_route_backward(const moga_shape& s, const void* X, const float* Wr, const float* logits,

@@ -1,11 +1,14 @@
-"""GPU parity of the backward of the routed group attention (bf16, d_head = 128) against the fp64
+"""GPU parity of the backward of the routed group attention (bf16 with d_head = 128 on the tensor
+cores, fp32 with d_head 64 / 128 on the fp32 ALUs) against the fp64
 oracle: the forward is run with the stage calls (which keep the sorted-order tensors and lse the
 backward needs), an upstream gradient dO is drawn, and dQ, dK, dV, dgate are compared.
 
 Tolerance: the kernels round the softmax weights, dS, the scaled upstream
 gradient and the sorted-order results to bf16 (2^-9 each) and accumulate in fp32, and the forward
 output they take as saved input is itself bf16: relative Frobenius error <= 1e-2 per gradient
-(measured ~3e-3), largest error <= 2^-5 of the tensor's largest magnitude."""
+(measured ~3e-3), largest error <= 2^-5 of the tensor's largest magnitude.  The fp32 path rounds
+nothing below fp32 (sums of a few hundred fp32 products, exp to ~2 ulp): relative Frobenius error
+<= 1e-5, largest error <= 2^-16 of the largest magnitude."""
 import numpy as np
 import pytest
 import torch
@@ -35,7 +38,8 @@ def _staged_forward(mb, cfg, inp):
     perm = torch.empty(cfg.B, T, dtype=torch.int32, device=dev)
     inv = torch.empty(cfg.B, cfg.N, cfg.k, dtype=torch.int32, device=dev)
     offsets = torch.empty(cfg.B, cfg.M + 1, dtype=torch.int32, device=dev)
-    Qp, Kp, Vp, Op = (torch.empty(cfg.B, cfg.H, T, cfg.D, dtype=torch.bfloat16, device=dev) for _ in range(4))
+    dt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    Qp, Kp, Vp, Op = (torch.empty(cfg.B, cfg.H, T, cfg.D, dtype=dt, device=dev) for _ in range(4))
     lse = torch.empty(cfg.B, cfg.H, T, dtype=torch.float32, device=dev)
     mb.moga_route(sh, inp["X"], inp["Wr"], inp["bias"], gid, gate, None, ws)
     mb.moga_permute(sh, gid, inp["Q"], inp["K"], inp["V"], perm, inv, offsets, Qp, Kp, Vp, ws)
@@ -49,6 +53,9 @@ CASES = [
     MogaConfig("b_top2", 2, 2, 700, 128, 128, 6, 2, "bf16", GATE_SOFTMAX_TOPK, 52),
     MogaConfig("b_ragged", 1, 3, 1111, 128, 128, 16, 1, "bf16", GATE_SOFTMAX_ALL, 53, zipf_bias=2.0),   # sizes 0, 1, ... hundreds
     MogaConfig("b_one_group", 1, 1, 385, 64, 128, 1, 1, "bf16", GATE_SOFTMAX_ALL, 54),
+    MogaConfig("f_top1_d64", 2, 2, 333, 64, 64, 4, 1, "f32", GATE_SOFTMAX_ALL, 55),
+    MogaConfig("f_top2_d128", 1, 2, 301, 64, 128, 5, 2, "f32", GATE_SOFTMAX_TOPK, 56),
+    MogaConfig("f_ragged_d64", 1, 3, 500, 64, 64, 16, 1, "f32", GATE_SOFTMAX_ALL, 57, zipf_bias=2.0),
 ]
 
 
@@ -57,7 +64,8 @@ def test_backward_matches_oracle(mb, cfg):
     inp = make_inputs(cfg, device="cuda")
     sh, fw = _staged_forward(mb, cfg, inp)
     g = torch.Generator(device="cuda").manual_seed(cfg.seed)
-    dO = torch.randn(cfg.B, cfg.H, cfg.N, cfg.D, generator=g, device="cuda").to(torch.bfloat16)
+    dO = torch.randn(cfg.B, cfg.H, cfg.N, cfg.D, generator=g, device="cuda").to(inp["Q"].dtype)
+    rel_bound, max_bound = (1e-2, 2.0 ** -5) if cfg.dtype == "bf16" else (1e-5, 2.0 ** -16)
     dQ, dK, dV = (torch.full_like(inp["Q"], float("nan")) for _ in range(3))
     dgate = torch.full((cfg.B, cfg.N, cfg.k), float("nan"), dtype=torch.float32, device="cuda")
     ws = mb.alloc_workspace(mb.moga_backward_workspace_bytes(sh))
@@ -72,8 +80,8 @@ def test_backward_matches_oracle(mb, cfg):
         err = np.abs(got - ref)
         rel = float(np.sqrt((err ** 2).sum() / max((ref ** 2).sum(), 1e-300)))
         print(f"{name}: rel fro {rel:.3e}  max err {err.max():.3e}  max |ref| {np.abs(ref).max():.3e}")
-        assert rel <= 1e-2, (name, rel)
-        assert err.max() <= 2.0 ** -5 * np.abs(ref).max() + 1e-6, (name, err.max())
+        assert rel <= rel_bound, (name, rel)
+        assert err.max() <= max_bound * np.abs(ref).max() + 1e-6, (name, err.max())
     # determinism: the same call twice gives the same bits
     dQ2, dK2, dV2 = (torch.empty_like(dQ) for _ in range(3))
     dg2 = torch.empty_like(dgate)
