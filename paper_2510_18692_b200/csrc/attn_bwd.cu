@@ -19,11 +19,14 @@
 // Computing the transposed products in the second launch keeps every A operand either K-major
 // in shared memory or row-per-lane in TMEM and every streamed tile usable as the MN-major B
 // operand of the accumulating MMAs: the same operand forms as the forward kernel, at the price of
-// seven GEMMs per tile pair instead of five.  The tensor pipe and the compute warps alternate
-// (one tile pair in flight); this kernel is the first correct form, not a tuned one.
-// TMEM: T0 [0,128) T1 [128,256) acc0 [256,384) acc1 [384,512); the bf16 results of the compute warps
-// overwrite columns [0,32) and [64,96) of the T region they were computed from (each half of the
-// threads writes inside the columns it has already read).
+// seven GEMMs per tile pair instead of five.
+// Overlap inside a CTA (one tile pair's T0 / T1 fill the TMEM beside the accumulators, so there is no
+// second buffer): the compute warps take T0 first (the exponentials, kept in registers) and release it,
+// so the next tile's T0 product runs while they work on T1; the accumulating MMAs of tile j and the T1
+// product of tile j+1 run while they take the exponentials of tile j+1.
+// TMEM: T0 [0,128) T1 [128,256) acc0 [256,384) acc1 [384,512).  Both bf16 results of the compute warps
+// go over T1: a thread that has read 32 of its T1 columns writes P over the first 16 of them and dS over
+// the other 16.
 #include <type_traits>
 
 #include "attn_common.cuh"
@@ -44,7 +47,7 @@ constexpr int kSmemR = 0;                        // resident pair
 constexpr int kSmemS = 2 * kTileBytes;           // streamed pairs
 constexpr int kSmemVec = kSmemS + NS * 2 * kTileBytes;   // 8 warps x (64 lse + 64 delta) floats
 constexpr int kSmemBar = kSmemVec + 8 * 128 * 4;
-constexpr int kNumBars = 2 + 2 * NS + 4;
+constexpr int kNumBars = 2 + 2 * NS + 6;
 constexpr int kSmemTotal = kSmemBar + 8 * kNumBars + 16;
 constexpr int kDynSmem = kSmemTotal + 1024;
 static_assert(kDynSmem <= 227 * 1024, "shared memory");
@@ -70,8 +73,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
   unsigned char* smem = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t sR = base + kSmemR, sS = base + kSmemS;
   const uint32_t bars = base + kSmemBar;
-  constexpr int R_FULL = 0, R_EMPTY = 1, S_FULL = 2, S_EMPTY = 2 + NS, T_FULL = 2 + 2 * NS, E_FULL = T_FULL + 1,
-                ACC_FULL = T_FULL + 2, ACC_EMPTY = T_FULL + 3;
+  constexpr int R_FULL = 0, R_EMPTY = 1, S_FULL = 2, S_EMPTY = 2 + NS, T0_FULL = 2 + 2 * NS, T1_FULL = T0_FULL + 1,
+                P_DONE = T0_FULL + 2, E_FULL = T0_FULL + 3, ACC_FULL = T0_FULL + 4, ACC_EMPTY = T0_FULL + 5;
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kSmemBar + 8 * kNumBars);
   volatile uint32_t* abort_flag = tmem_slot + 1;
@@ -86,7 +89,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
       mbar_init(bar(S_FULL + i), 1);
       mbar_init(bar(S_EMPTY + i), 1);
     }
-    mbar_init(bar(T_FULL), 1);
+    mbar_init(bar(T0_FULL), 1);
+    mbar_init(bar(T1_FULL), 1);
+    mbar_init(bar(P_DONE), 2 * kTile);
     mbar_init(bar(E_FULL), 2 * kTile);
     mbar_init(bar(ACC_FULL), 1);
     mbar_init(bar(ACC_EMPTY), 2 * kTile);
@@ -155,13 +160,14 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
           mma_ss(tmem + t * kTile, ra + o, sb + o, hi, idesc_t, kk > 0);
         }
       };
-      // acc[a] (+)= E[e] S[t]   (E: bf16, streamed rows 0-63 in columns [0,32) of T[e], rows 64-127 in [64,96))
+      // acc[a] (+)= E[e] S[t]   (E[e]: bf16 over T1; the 16 streamed rows of k-step kk sit in 8 columns
+      // of the thread half kk / 4, its chunk (kk % 4) / 2; P first, dS 16 columns on)
       auto issue_acc = [&](int a, int e, int t, uint32_t stage, bool accumulate) {
         const uint32_t vb = desc_lo(stage + t * kTileBytes, kBoxBytes);
 #pragma unroll
         for (int kk = 0; kk < kTile / 16; ++kk)
-          mma_ts(tmem + 256 + a * 128, tmem + e * kTile + (kk / 4) * 64 + (kk % 4) * 8, vb + ((kk * 2048) >> 4), hi,
-                 idesc_a, (accumulate || kk > 0) ? 1u : 0u);
+          mma_ts(tmem + 256 + a * 128, tmem + kTile + (kk / 4) * 64 + ((kk % 4) / 2) * 32 + (kk % 2) * 8 + e * 16,
+                 vb + ((kk * 2048) >> 4), hi, idesc_a, (accumulate || kk > 0) ? 1u : 0u);
       };
       uint32_t nit = 0, ns = 0, nt = 0;
       bool ok = true;
@@ -170,15 +176,29 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
         const int ntiles = (it.khi - it.klo + kTile - 1) / kTile;
         ok = wait(R_FULL, nit & 1u, 3);
         if (!ok) break;
+        // first tile: both products.  T0 is free (P_DONE of the previous item's last tile was waited
+        // for below); T1 held that tile's P / dS, whose MMAs were issued before these (the pipe keeps issue order).
+        ok = wait(S_FULL + ns % NS, (ns / NS) & 1u, 4);
+        if (!ok) break;
+        tc_fence_after();
+        issue_t(0, sS + (ns % NS) * 2 * kTileBytes);
+        tc_commit(bar(T0_FULL));
+        issue_t(1, sS + (ns % NS) * 2 * kTileBytes);
+        tc_commit(bar(T1_FULL));
+        if (ntiles == 1) tc_commit(bar(R_EMPTY));
         for (int j = 0; j < ntiles && ok; ++j, ++ns, ++nt) {
-          const int s = ns % NS;
-          const uint32_t stage = sS + s * 2 * kTileBytes;
-          ok = wait(S_FULL + s, (ns / NS) & 1u, 4);
+          const uint32_t stage = sS + (ns % NS) * 2 * kTileBytes;
+          const uint32_t next = sS + ((ns + 1) % NS) * 2 * kTileBytes;
+          const bool more = j + 1 < ntiles;
+          ok = wait(P_DONE, nt & 1u, 9);                  // T0 of tile j has been read
           if (!ok) break;
-          tc_fence_after();
-          issue_t(0, stage);
-          issue_t(1, stage);
-          tc_commit(bar(T_FULL));
+          if (more) {
+            ok = wait(S_FULL + (ns + 1) % NS, ((ns + 1) / NS) & 1u, 4);
+            if (!ok) break;
+            tc_fence_after();
+            issue_t(0, next);
+            tc_commit(bar(T0_FULL));
+          }
           ok = wait(E_FULL, nt & 1u, 5);
           if (!ok) break;
           if (j == 0) {
@@ -192,10 +212,13 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
             issue_acc(0, 0, 1, stage, j > 0);             // dV += P^T dO
             issue_acc(1, 1, 0, stage, j > 0);             // dK += dS^T Q
           }
-          tc_commit(bar(S_EMPTY + s));
-          if (j + 1 == ntiles) {
+          tc_commit(bar(S_EMPTY + ns % NS));
+          if (more) {
+            issue_t(1, next);                             // over the P / dS the MMAs above read
+            tc_commit(bar(T1_FULL));
+            if (j + 2 == ntiles) tc_commit(bar(R_EMPTY));
+          } else {
             tc_commit(bar(ACC_FULL));
-            tc_commit(bar(R_EMPTY));
           }
         }
       }
@@ -237,29 +260,21 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
           }
           __syncwarp();
         }
-        ok = __all_sync(0xffffffffu, wait(T_FULL, nt & 1u, 7));
+        ok = __all_sync(0xffffffffu, wait(T0_FULL, nt & 1u, 7));
         if (!ok) break;
         tc_fence_after();
-        // p = 2^(t0 * scale_log2 - lse * log2e),  ds = p * (t1 * scale - delta * scale): packed fp32 pairs.
+        // p = 2^(t0 * scale_log2 - lse * log2e), kept in registers; T0 is then free for the next tile.
         // A tile that reaches past the group's end takes the variant that zeroes those columns' p.
         const float2 sl2 = make_float2(scale_log2, scale_log2), sc2 = make_float2(scale, scale);
-        auto chunk = [&](int ch, auto masked) {
-          uint32_t t0[32], t1[32];
+        float2 p[32];
+        auto weights = [&](int ch, auto masked) {
+          uint32_t t0[32];
           tmem_ld32(tT0 + ch * 32, t0);
-          tmem_ld32(tT1 + ch * 32, t1);
           tmem_wait_ld();
-          uint32_t ep[16], ed[16];
 #pragma unroll
           for (int c = 0; c < 32; c += 2) {
             const int lc = ch * 32 + c;
-            float2 nl2, nds;                          // minus lse * log2e, minus delta * scale, of the two columns
-            if (Mode == kModeQ) {
-              nl2 = make_float2(row_lse, row_lse);
-              nds = make_float2(row_delta, row_delta);
-            } else {
-              nl2 = *reinterpret_cast<const float2*>(wvec + lc);
-              nds = *reinterpret_cast<const float2*>(wvec + 64 + lc);
-            }
+            const float2 nl2 = Mode == kModeQ ? make_float2(row_lse, row_lse) : *reinterpret_cast<const float2*>(wvec + lc);
             const float2 x = __ffma2_rn(make_float2(__uint_as_float(t0[c]), __uint_as_float(t0[c + 1])), sl2, nl2);
             float2 pe = make_float2(ex2(x.x), ex2(x.y));
             if (decltype(masked)::value) {
@@ -267,24 +282,44 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap mapR0, const __grid_constant
               pe.x = col < ncols ? pe.x : 0.f;
               pe.y = col + 1 < ncols ? pe.y : 0.f;
             }
+            p[lc >> 1] = pe;
+          }
+        };
+        if (ncols < kTile) {
+          weights(0, std::true_type{});
+          weights(1, std::true_type{});
+        } else {
+          weights(0, std::false_type{});
+          weights(1, std::false_type{});
+        }
+        tc_fence_before();
+        mbar_arrive(bar(P_DONE));
+        ok = __all_sync(0xffffffffu, wait(T1_FULL, nt & 1u, 10));
+        if (!ok) break;
+        tc_fence_after();
+        // ds = p * (t1 * scale - delta * scale).  Chunk ch of this thread's T1 columns has been read when
+        // its results are written: P over the chunk's first 16 columns, dS over its last 16.
+#pragma unroll
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t t1[32];
+          tmem_ld32(tT1 + ch * 32, t1);
+          tmem_wait_ld();
+          uint32_t ep[16], ed[16];
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) {
+            const int lc = ch * 32 + c;
+            const float2 nds = Mode == kModeQ ? make_float2(row_delta, row_delta)
+                                              : *reinterpret_cast<const float2*>(wvec + 64 + lc);
             const float2 u = __ffma2_rn(make_float2(__uint_as_float(t1[c]), __uint_as_float(t1[c + 1])), sc2, nds);
+            const float2 pe = p[lc >> 1];
             const float2 ds = __fmul2_rn(pe, u);
             __nv_bfloat162 a = __floats2bfloat162_rn(pe.x, pe.y);
             __nv_bfloat162 b = __floats2bfloat162_rn(ds.x, ds.y);
             ep[c >> 1] = *reinterpret_cast<uint32_t*>(&a);
             ed[c >> 1] = *reinterpret_cast<uint32_t*>(&b);
           }
-          // chunk ch of this thread's columns has been read: its bf16 results overwrite the first
-          // 16 (ch = 0) / next 16 columns of the same 64-column range
-          if (Mode == kModeKV) tmem_st16(tT0 + ch * 16, ep);
-          tmem_st16(tT1 + ch * 16, ed);
-        };
-        if (ncols < kTile) {
-          chunk(0, std::true_type{});
-          chunk(1, std::true_type{});
-        } else {
-          chunk(0, std::false_type{});
-          chunk(1, std::false_type{});
+          if (Mode == kModeKV) tmem_st16(tT1 + ch * 32, ep);
+          tmem_st16(tT1 + ch * 32 + 16, ed);
         }
         tmem_wait_st();
         tc_fence_before();
