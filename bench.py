@@ -40,18 +40,31 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes of the attention kernel / its algorithmic bytes, from the ncu capture of the
 # clip-sized case (traffic grows with T*H: every Q/K/V/O byte crosses DRAM once).  The figure
 # belongs to one version of the kernel source: when the source's hash differs, traffic is null.
-ATTN_TRAFFIC = {"ratio": 0.9565, "source_sha16": "6a7a8dee240eb5b1"}
+ATTN_TRAFFIC = {"duo": {"file": "attn_bf16_duo.cu", "ratio": None, "source_sha16": None},
+                "single": {"file": "attn_bf16.cu", "ratio": 0.9565, "source_sha16": "6a7a8dee240eb5b1"}}
 
 
-def attn_traffic_ratio():
+def attn_traffic_ratio(kernel):
     import hashlib
-    path = os.path.join(ROOT, "paper_2510_18692_b200", "csrc", "attn_bf16.cu")
+    rec = ATTN_TRAFFIC.get(kernel)
+    if rec is None:
+        return None
+    path = os.path.join(ROOT, "paper_2510_18692_b200", "csrc", rec["file"])
     try:
         with open(path, "rb") as f:
             sha = hashlib.sha256(f.read()).hexdigest()[:16]
     except OSError:
         return None
-    return ATTN_TRAFFIC["ratio"] if sha == ATTN_TRAFFIC["source_sha16"] else None
+    return rec["ratio"] if sha == rec["source_sha16"] else None
+
+
+def attn_kernel_name(cfg, choice):
+    """Which group-attention kernel a forward of cfg runs under --attn-kernel `choice`."""
+    if cfg.dtype != "bf16":
+        return "alu"
+    if cfg.D != 128 or choice == "single":
+        return "single"
+    return "pair" if choice == "pair" else "duo"
 
 
 def schedule_tail(offsets_np, H, n_ctas=148, qblock=256, tile_n=128):
@@ -78,12 +91,13 @@ def schedule_tail(offsets_np, H, n_ctas=148, qblock=256, tile_n=128):
     return float(load.max() / load.mean()) if load.mean() > 0 else 1.0
 
 
-def kernels_per_forward(cfg):
+def kernels_per_forward(cfg, attn_kernel="duo"):
     """Kernels one moga_forward launches: router (bf16: weight split + tensor-core router; fp32: one
-    ALU kernel), 3 sort kernels, gather, attention (bf16: schedule + attention), and the gated
-    unpermute unless the bf16 top-1 attention epilogue already wrote token order."""
+    ALU kernel), 3 sort kernels, gather, attention (bf16: schedule + attention, plus the launch of the
+    exact kernel over the list of handed-over items when the default or the CTA-pair kernel runs),
+    and the gated unpermute unless the bf16 top-1 attention epilogue already wrote token order."""
     if cfg.dtype == "bf16":
-        return 2 + 3 + 1 + 2 + (1 if cfg.k > 1 else 0)
+        return 2 + 3 + 1 + (3 if attn_kernel in ("duo", "pair") else 2) + (1 if cfg.k > 1 else 0)
     return 1 + 3 + 1 + 1 + 1
 
 
@@ -275,8 +289,9 @@ def main():
                          "branches and their mean; 'backward' times moga_backward (gradients of the group attention and "
                          "the gates) after a staged forward of the config")
     ap.add_argument("--attn-kernel", default="auto", choices=["auto", "single", "pair"],
-                    help="bf16 group-attention kernel (moga_set_attn_kernel): the one-CTA kernel (default) or the "
-                         "CTA-pair kernel, for A/B runs and profiles")
+                    help="bf16 group-attention kernel (moga_set_attn_kernel): auto (two softmax threads per row where "
+                         "the launch allows it), the one-thread-per-row kernel, or the CTA-pair kernel, for A/B runs "
+                         "and profiles")
     ap.add_argument("--topk-epilogue", default="staged", choices=["staged", "add"],
                     help="bf16 top-2 output path (moga_set_fused_topk): permuted output + unpermute (default) or "
                          "gate * row added into token order by the attention epilogue")
@@ -401,7 +416,8 @@ def main():
                                      "frac_tensor_sustained": attn_tflops / peaks["bf16_tflops_sustained"],
                                      # time x clock: compares boxes whose power cap settles at different clocks
                                      "ms_x_sm_mhz": None if not mhz else stage["group_attn"] * mhz})
-    ratio = attn_traffic_ratio() if cfg.dtype == "bf16" else None
+    akern = attn_kernel_name(cfg, args.attn_kernel)
+    ratio = attn_traffic_ratio(akern)
     out = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "ms_per_step_mean": ms_mean,
@@ -409,11 +425,11 @@ def main():
         "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic", "config": config_dict(cfg),
         "route_kernel": "tensor" if cfg.dtype == "bf16" else "alu",
-        "attn_kernel": ("pair" if args.attn_kernel == "pair" and cfg.D == 128 else "single") if cfg.dtype == "bf16" else "alu",
+        "attn_kernel": akern,
         "topk_epilogue": args.topk_epilogue if (cfg.dtype == "bf16" and cfg.k == 2) else None,
         "ms_per_layer_head_batch": ms / (cfg.B * cfg.H), "useful_tflop_per_step": flops / 1e12,
         "group_sizes": {"min": int(sizes.min()), "max": int(sizes.max()), "empty": int((sizes == 0).sum())},
-        "stages": stages_out, "gpu_launches": kernels_per_forward(cfg) * args.steps, "clocks": clk,
+        "stages": stages_out, "gpu_launches": kernels_per_forward(cfg, akern) * args.steps, "clocks": clk,
         "schedule_tail": schedule_tail(offsets.cpu().numpy(), cfg.H) if cfg.dtype == "bf16" else None,
     }
     if cfg.dtype == "bf16":
@@ -594,7 +610,7 @@ def run_head_sharded(mb, cfg, dev, args, rank, world):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "strong", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
             "config": dict(config_dict(cfg), sharding="tokens for routing, heads for attention; one all-gather of (gid, gate)"),
-            "gpu_launches": kernels_per_forward(cfg) * args.steps,
+            "gpu_launches": kernels_per_forward(cfg, attn_kernel_name(cfg, args.attn_kernel)) * args.steps,
             "ms_per_layer_head_batch": ms * world / (cfg.B * cfg.H),
             "clocks": clk}))
     return 0

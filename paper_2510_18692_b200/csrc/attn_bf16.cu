@@ -548,18 +548,22 @@ moga_status launch_one(const Problem& p, cudaStream_t st) {
   return MOGA_OK;
 }
 
-// Which kernel serves a launch.  The one-CTA kernel is the default for every shape: measured on
-// groups of ~17,500 rows it runs at 1,150-1,160 TFLOP/s against 935 for the CTA-pair kernel (same
-// box, alternating runs).  The pair kernel halves the K/V bytes each SM stages and reads per
-// flop, but issuing an M = 256, N = 128 instruction for two SMs keeps the issuing thread about as
-// long as the instruction runs, so its waits are no longer hidden behind queued MMAs and the
-// tensor pipe idles 55 % of the cycles.  It stays selectable (moga_set_attn_kernel) for d_head = 128
-// launches that have the redo scratch.
+// Which kernel serves a launch.  Default for d_head = 128 launches that have the redo scratch and
+// store their rows (sorted order or the top-1 scatter): the kernel with two softmax threads per row
+// (attn_bf16_duo.cu), followed by this file's kernel over the items it listed; measured on groups of
+// ~17,500 rows, same box, alternating runs: 1,202 TFLOP/s against 1,157 for this file's kernel alone.
+// Everything else (d_head = 64, static groups, the adding epilogue) runs this file's kernel.
+// The CTA-pair kernel (935 TFLOP/s on the same case) halves the K/V bytes each SM stages and reads
+// per flop, but issuing an M = 256, N = 128 instruction for two SMs keeps the issuing thread about as
+// long as the instruction runs, so its waits are no longer hidden behind queued MMAs and the tensor
+// pipe idles 55 % of the cycles.  It stays selectable (moga_set_attn_kernel).
 int g_attn_kernel = MOGA_ATTN_AUTO;
 
 moga_status launch_any(int D, const Problem& p, cudaStream_t st) {
-  const bool pair = D == 128 && p.redo != nullptr && p.epi == kEpiDefault && g_attn_kernel == MOGA_ATTN_PAIR;
-  return pair ? launch_pair(p, st) : launch_single(D, p, st);
+  const bool listable = D == 128 && p.redo != nullptr && p.epi == kEpiDefault;
+  if (listable && g_attn_kernel == MOGA_ATTN_PAIR) return launch_pair(p, st);
+  if (listable && g_attn_kernel == MOGA_ATTN_AUTO) return launch_duo(p, st);
+  return launch_single(D, p, st);
 }
 
 // Routed groups: offsets [B, M+1] serve queries and keys alike; scratch from the workspace layout.

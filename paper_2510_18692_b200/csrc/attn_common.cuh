@@ -112,8 +112,8 @@ struct Problem {
   float* lse;
   Groups grp;
   int32_t *order, *prefix;   // scratch: B*G and B*G + 1 int32
-  int32_t* redo;             // scratch of the CTA-pair kernel (items for the exact path): int32
-                             // [4 + 2 * max_items_256]; nullptr: the launch cannot use that kernel
+  int32_t* redo;             // scratch of the kernels that hand items to the exact path: int32
+                             // [4 + 2 * max_items_256]; nullptr: the launch cannot use those kernels
   uint32_t* header;          // device status word
   Scatter sc;
   int epi;                   // kEpiDefault / kEpiList / kEpiMean3 (the latter two: one-CTA kernel, D = 128)
@@ -129,6 +129,7 @@ inline long long max_items_256(const Problem& p) {
 // query block
 moga_status launch_single(int D, const Problem& p, cudaStream_t st);   // 256 query rows per CTA
 moga_status launch_pair(const Problem& p, cudaStream_t st);            // D = 128, 256 query rows per CTA pair
+moga_status launch_duo(const Problem& p, cudaStream_t st);             // D = 128, two softmax threads per row
 // D = 128: the one-CTA kernel over the items listed in p.redo (their schedule is already in place)
 moga_status launch_single_redo(const Problem& p, cudaStream_t st);
 

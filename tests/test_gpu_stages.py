@@ -245,8 +245,9 @@ PAIR_SIZES = [
 
 @pytest.mark.parametrize("sizes", PAIR_SIZES, ids=lambda s: "g" + "_".join(map(str, s[:4])))
 def test_group_attn_pair_kernel(mb, sizes):
-    """The CTA-pair kernel (512 query rows per pair of SMs, d_head = 128), forced for every group
-    size, against the oracle and against the one-CTA kernel; then the automatic choice."""
+    """The three tensor-core kernels for d_head = 128 (the CTA-pair kernel, the one-CTA kernel with one
+    softmax thread per row, and the default with two softmax threads per row), each forced for
+    every group size, against the oracle and against each other."""
     H, B, D = 2, 2, 128
     case = grouped_case(sizes, H, D, "bf16", seed=len(sizes) + 7, B=B)
     T, M = case["T"], len(sizes)
@@ -259,7 +260,7 @@ def test_group_attn_pair_kernel(mb, sizes):
                            np.ones((B, T, 1)), case["offsets"], case["perm"], scale)
     outs = {}
     try:
-        for mode in (mb.MOGA_ATTN_PAIR, mb.MOGA_ATTN_SINGLE):
+        for mode in (mb.MOGA_ATTN_PAIR, mb.MOGA_ATTN_SINGLE, mb.MOGA_ATTN_AUTO):
             mb.moga_set_attn_kernel(mode)
             Op = torch.full_like(case["Q"], float("nan"))
             lse = torch.empty(B, H, T, dtype=torch.float32, device="cuda")
@@ -270,9 +271,12 @@ def test_group_attn_pair_kernel(mb, sizes):
     finally:
         mb.moga_set_attn_kernel(mb.MOGA_ATTN_AUTO)
     # same arithmetic per row in both kernels: expected equal to the last bit; at the least very close
-    a, b = outs[mb.MOGA_ATTN_PAIR], outs[mb.MOGA_ATTN_SINGLE]
-    assert (a[0].float() - b[0].float()).abs().max().item() <= 2.0 ** -7 * b[0].float().abs().max().item() + 1e-6
-    assert (a[1] - b[1]).abs().max().item() <= 1e-3
+    b = outs[mb.MOGA_ATTN_SINGLE]
+    for mode in (mb.MOGA_ATTN_PAIR, mb.MOGA_ATTN_AUTO):
+        a = outs[mode]
+        assert (a[0].float() - b[0].float()).abs().max().item() <= 2.0 ** -7 * b[0].float().abs().max().item() + 1e-6
+        assert (a[1] - b[1]).abs().max().item() <= 1e-3
+    a = outs[mb.MOGA_ATTN_PAIR]
     q, k_ = case["Q"].double().cpu(), case["K"].double().cpu()
     for g in range(M):
         lo, hi = case["offsets"][0, g], case["offsets"][0, g + 1]
@@ -357,11 +361,12 @@ def test_group_attn_neighbour_group_does_not_leak(mb, dtype):
     assert torch.equal(outs[0], outs[1])
 
 
-@pytest.mark.parametrize("kernel", ["single", "pair"])
+@pytest.mark.parametrize("kernel", ["single", "pair", "auto"])
 @pytest.mark.parametrize("grow", [3.0, 24.0])
 def test_group_attn_growing_scores_bf16(mb, grow, kernel):
-    """Both kernels: the one-CTA kernel changes the reference inside the row; the CTA-pair kernel
-    hands such items to the one-CTA kernel's exact path afterwards.
+    """All three kernels: the one-CTA kernel with one thread per row changes the reference inside the
+    row; the default (two threads per row) and the CTA-pair kernel hand such items to that kernel's
+    exact path afterwards.
     Keys late in each group are scaled up, so later K/V tiles hold scores far above the
     first tile's maximum: x3 stays on the kernel's fixed-reference path with large positive
     exponents, x24 overflows it and forces the mid-row change of reference.  Outputs are
@@ -378,7 +383,7 @@ def test_group_attn_growing_scores_bf16(mb, grow, kernel):
     Op = torch.full_like(case["Q"], float("nan"))
     lse = torch.empty(1, 2, case["T"], dtype=torch.float32, device="cuda")
     ws = mb.alloc_workspace(mb.moga_scratch_bytes(sh))
-    mb.moga_set_attn_kernel(mb.MOGA_ATTN_PAIR if kernel == "pair" else mb.MOGA_ATTN_SINGLE)
+    mb.moga_set_attn_kernel({"pair": mb.MOGA_ATTN_PAIR, "single": mb.MOGA_ATTN_SINGLE, "auto": mb.MOGA_ATTN_AUTO}[kernel])
     try:
         mb.moga_group_attn(sh, case["Q"], case["K"], case["V"], torch.from_numpy(case["offsets"]).cuda(), Op,
                            lse, ws)
