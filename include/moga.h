@@ -361,14 +361,19 @@ moga_status moga_route_backward(const moga_shape* s, const void* X, const float*
 
 /*
  * Choice of the bf16 group-attention kernel (the paper has no counterpart: a tuning and test
- * switch).  Two kernels compute Eq. 1 inside the groups on the tensor cores.  The default
- * (MOGA_ATTN_AUTO, same as MOGA_ATTN_SINGLE) gives a block of 256 query rows to one SM.
- * MOGA_ATTN_PAIR gives 256 query rows to a pair of SMs that issue every tensor-core
- * instruction together and each stage half of every K/V tile (d_head = 128, routed launches
- * only; other launches keep the default).  The pair kernel is correct on every shape but
- * measured slower (see the kernel selection comment in csrc/attn_bf16.cu); it is kept as an
- * option.  Process-wide, not thread-safe against concurrent launches; returns
- * MOGA_ERR_INVALID_ARG for another value.
+ * switch).  Three kernels compute Eq. 1 inside the groups on the tensor cores; all give a block
+ * of 256 query rows (two 128-row tiles) to one work item.
+ * MOGA_ATTN_AUTO (default): for d_head = 128, routed groups and a storing epilogue, the kernel
+ * with two softmax threads per query row, which keeps the first key tile's row maximum as the
+ * reference and hands any item whose scores outgrow it by 2^40 to the exact kernel; every other
+ * launch runs MOGA_ATTN_SINGLE.
+ * MOGA_ATTN_SINGLE: one SM per item, one softmax thread per row, the reference raised inside
+ * the row when needed (the exact kernel).
+ * MOGA_ATTN_PAIR: a pair of SMs per item that issue every tensor-core instruction together and
+ * each stage half of every K/V tile (d_head = 128, routed launches only); correct on every shape
+ * but measured slower (see the kernel selection comment in csrc/attn_bf16.cu); kept as an option.
+ * Process-wide, not thread-safe against concurrent launches; returns MOGA_ERR_INVALID_ARG for
+ * another value.
  */
 typedef enum { MOGA_ATTN_AUTO = 0, MOGA_ATTN_SINGLE = 1, MOGA_ATTN_PAIR = 2 } moga_attn_kernel;
 moga_status moga_set_attn_kernel(int32_t mode);
