@@ -225,3 +225,38 @@ def test_single_token_and_no_token(mb):
     mb.moga_unpermute(sh, None, None, None, None)
     torch.cuda.synchronize()
     assert torch.all(off == 0)
+
+
+def test_forward_replays_from_a_cuda_graph(mb):
+    """Every launch of moga_forward goes to the caller's stream and none of its host code
+    synchronises, so the call can be captured once and replayed: the replay on new input values
+    (same buffers) gives the bits of a direct call."""
+    cfg = MogaConfig("graph", 1, 3, 1500, 256, 128, 6, 1, "bf16", GATE_SOFTMAX_ALL, 31)
+    inp = make_inputs(cfg, device="cuda")
+    sh = mb.make_shape(cfg)
+    ws = mb.alloc_workspace(mb.moga_workspace_bytes(sh))
+    O = torch.zeros_like(inp["Q"])
+    args = (sh, inp["X"], inp["Wr"], inp["bias"], inp["Q"], inp["K"], inp["V"], O, ws)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        mb.moga_forward(*args)                    # warm-up outside the capture (function attributes, tensor-map entry point)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        mb.moga_forward(*args)
+    # new values in the captured buffers
+    fresh = make_inputs(MogaConfig("graph2", 1, 3, 1500, 256, 128, 6, 1, "bf16", GATE_SOFTMAX_ALL, 32), device="cuda")
+    for name in ("X", "Q", "K", "V"):
+        inp[name].copy_(fresh[name])
+    O.fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    assert mb.moga_last_device_status(ws) == (0, 0)
+    replayed = O.clone()
+    O.fill_(float("nan"))
+    mb.moga_forward(*args)
+    torch.cuda.synchronize()
+    assert torch.isfinite(replayed.float()).all()
+    assert torch.equal(replayed, O)
