@@ -260,3 +260,24 @@ def test_forward_replays_from_a_cuda_graph(mb):
     torch.cuda.synchronize()
     assert torch.isfinite(replayed.float()).all()
     assert torch.equal(replayed, O)
+
+
+def test_forward_top1_with_scores_that_outgrow_the_first_tile(mb):
+    """Fused top-1 forward (attention epilogue scatters gate * row to token order) on keys that grow
+    along the sequence: late key tiles of every group hold scores far above the first tile's
+    maximum, so the default d_head = 128 kernel hands those items to the exact kernel, which must
+    overwrite their rows in token order with the same gates.  Relative bounds: a few keys dominate
+    each row, so outputs are O(1)."""
+    cfg = MogaConfig("grow", 1, 2, 2600, 128, 128, 4, 1, "bf16", GATE_SOFTMAX_ALL, 41)
+    inp = make_inputs(cfg, device="cuda")
+    inp["K"][:, :, cfg.N // 3:] *= 24.0
+    host = {k: to_np32(v) for k, v in inp.items()}
+    O, gid, gate, perm, offsets = run_forward(mb, cfg, inp)
+    o_off, o_perm, _ = oracle.sort(gid.cpu().numpy(), cfg.M)
+    assert np.array_equal(perm.cpu().numpy(), o_perm)
+    want = oracle.attn_all(host["Q"], host["K"], host["V"], gid.cpu().numpy(), gate.double().cpu().numpy(),
+                           o_off, o_perm, cfg.scale)
+    got = O.float().cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(got))
+    assert np.linalg.norm(got - want) / np.linalg.norm(want) < 1e-2
+    assert np.abs(got - want).max() <= 2.0 ** -6 * np.abs(want).max()
