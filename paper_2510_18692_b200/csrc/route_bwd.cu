@@ -183,58 +183,82 @@ route_dx_kernel(const float* __restrict__ dr, const float* __restrict__ Wr, XT* 
 }
 
 // part[slab, c, i] = sum over the slab's tokens of X[t, c] dr[t, i], for the block's 128 channels.
-// Thread (lane = channel quad, warp = group of MC = ceil(M / 8) logit columns) owns 4 channels x MC
-// columns; per token it reads 4 channels of X and MC values of dr (the same for the whole warp).
-// (First form: the X loads, eight bytes per thread and token with four in flight, are latency-bound;
-// measured 10-15 TFLOP/s fp32 at the minute-long size (25-39 ms, 3-5 % of the backward step).  Wider column blocks per thread were tried and
-// were slower at one block per SM; staging X through shared memory with cp.async is the next step.)
-template <typename XT>
+// A thread owns 4 channels (lane = channel quad) x COLS logit columns: 4 * COLS accumulators, so that a
+// token costs it one 8- or 16-byte load of X and 4 * COLS FMAs against dr values broadcast from shared
+// memory.  The 8 warps of a block split into ceil(M / COLS) column blocks (1, 2 or 4: X is read once per
+// column block); the warps of a column block take the tile's tokens in turn and their sums are added at the
+// end of the slab in warp order through shared memory: a fixed order, no atomics.  Measured at the
+// minute-long size (M = 32): 9.0 ms with two 16-column blocks, 14.7 ms with one 32-column block (180
+// registers, one block per SM), 17.1 ms for the first form (each warp a column group, X read by all eight).
+template <typename XT, int COLS>
 __global__ void __launch_bounds__(256)
 route_dw_partial_kernel(const XT* __restrict__ X, const float* __restrict__ dr, float* __restrict__ part,
                         long long tokens, int C, int M) {
-  constexpr int kTokTile = 64;
+  constexpr int kTokTile = 128;
+  // dr of the tile's tokens; after the last tile the same memory holds the 128 x M sums being added
   __shared__ __align__(16) float sdr[kTokTile][kMaxM];
+  static_assert(kTokTile * kMaxM >= kWcChunk * kMaxM, "the sums fit where the dr tile was");
   const int slab = blockIdx.y;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int c = blockIdx.x * kWcChunk + lane * 4;
-  const int MC = (M + 7) / 8, i0 = warp * MC;
+  const int ncb = (M + COLS - 1) / COLS;           // 1, 2 or 4 (the launcher picks COLS so)
+  const int wpc = 8 / ncb;                         // warps per column block
+  const int cb = warp / wpc, wl = warp % wpc;
+  const int i0 = cb * COLS;
   const long long per = (tokens + kSlabs - 1) / kSlabs;
   const long long ta = (long long)slab * per, tb = min(tokens, ta + per);
-  float acc[4][kMaxM / 8];
+  float acc[4][COLS];
 #pragma unroll
   for (int u = 0; u < 4; ++u)
 #pragma unroll
-    for (int i = 0; i < kMaxM / 8; ++i) acc[u][i] = 0.f;
+    for (int i = 0; i < COLS; ++i) acc[u][i] = 0.f;
   for (long long t0 = ta; t0 < tb; t0 += kTokTile) {
     __syncthreads();
-    for (int idx = threadIdx.x; idx < kTokTile * M; idx += 256) {
-      const int tt = idx / M, i = idx % M;
-      sdr[tt][i] = t0 + tt < tb ? dr[(t0 + tt) * M + i] : 0.f;
+    const int mp = ncb * COLS;                     // columns the threads read (zero beyond M)
+    for (int idx = threadIdx.x; idx < kTokTile * mp; idx += 256) {
+      const int tt = idx / mp, i = idx % mp;
+      sdr[tt][i] = (t0 + tt < tb && i < M) ? dr[(t0 + tt) * M + i] : 0.f;
     }
     __syncthreads();
-    if (c < C && i0 < M) {
+    if (c < C) {
       const int nt = (int)min((long long)kTokTile, tb - t0);
 #pragma unroll 4
-      for (int tt = 0; tt < nt; ++tt) {
+      for (int tt = wl; tt < nt; tt += wpc) {
         float x[4];
         load4(X + (t0 + tt) * C + c, x);
 #pragma unroll
-        for (int i = 0; i < kMaxM / 8; ++i) {
-          if (i < MC) {
-            const float dv = i0 + i < M ? sdr[tt][i0 + i] : 0.f;
+        for (int i = 0; i < COLS; i += 4) {
+          const float4 dv = *reinterpret_cast<const float4*>(&sdr[tt][i0 + i]);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) acc[u][i] = fmaf(x[u], dv, acc[u][i]);
+          for (int u = 0; u < 4; ++u) {
+            acc[u][i] = fmaf(x[u], dv.x, acc[u][i]);
+            acc[u][i + 1] = fmaf(x[u], dv.y, acc[u][i + 1]);
+            acc[u][i + 2] = fmaf(x[u], dv.z, acc[u][i + 2]);
+            acc[u][i + 3] = fmaf(x[u], dv.w, acc[u][i + 3]);
           }
         }
       }
     }
   }
-  if (c < C)
+  // the column block's warps add their sums in warp order
+  __syncthreads();
+  float* r = &sdr[0][0] + (cb * kWcChunk + lane * 4) * COLS;
+  for (int w = 0; w < wpc; ++w) {
+    __syncthreads();
+    if (wl == w) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int i = 0; i < COLS; ++i) r[u * COLS + i] = w == 0 ? acc[u][i] : r[u * COLS + i] + acc[u][i];
+    }
+  }
+  __syncthreads();
+  if (wl == 0 && c < C)
 #pragma unroll
     for (int u = 0; u < 4; ++u)
 #pragma unroll
-      for (int i = 0; i < kMaxM / 8; ++i)
-        if (i < MC && i0 + i < M) part[((size_t)slab * C + c + u) * M + i0 + i] = acc[u][i];
+      for (int i = 0; i < COLS; ++i)
+        if (i0 + i < M) part[((size_t)slab * C + c + u) * M + i0 + i] = r[u * COLS + i];
 }
 
 // dWr[c, i] = sum over slabs (in order) of part[slab, c, i];  dbias[i] = sum over blocks of colsum
@@ -252,6 +276,16 @@ route_dw_reduce_kernel(const float* __restrict__ part, float* __restrict__ dWr, 
     for (int b = 0; b < nblk; ++b) acc += colsum[(size_t)b * M + threadIdx.x];
     dbias[threadIdx.x] = acc;
   }
+}
+
+// COLS: 8 for M <= 8, else 16 (1, 2 or 4 column blocks for M <= 16, 32, 64)
+template <typename XT>
+void launch_dw_partial(const XT* X, const float* dr, float* part, long long tokens, int C, int M, dim3 grid,
+                       cudaStream_t st) {
+  if (M <= 8)
+    route_dw_partial_kernel<XT, 8><<<grid, 256, 0, st>>>(X, dr, part, tokens, C, M);
+  else
+    route_dw_partial_kernel<XT, 16><<<grid, 256, 0, st>>>(X, dr, part, tokens, C, M);
 }
 
 }  // namespace
@@ -287,8 +321,7 @@ moga_status launch_route_backward(const moga_shape& s, const void* X, const floa
       route_dx_kernel<__nv_bfloat16><<<(unsigned)((tokens + kDxTok - 1) / kDxTok), 256, dx_smem_bytes, st>>>(
           dr, Wr, static_cast<__nv_bfloat16*>(dX), tokens, s.C, s.M);
     }
-    route_dw_partial_kernel<__nv_bfloat16><<<wgrid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(X), dr, part,
-                                                                  tokens, s.C, s.M);
+    launch_dw_partial(static_cast<const __nv_bfloat16*>(X), dr, part, tokens, s.C, s.M, wgrid, st);
   } else {
     if (dX) {
       MOGA_CUDA_OK(cudaFuncSetAttribute(route_dx_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -296,7 +329,7 @@ moga_status launch_route_backward(const moga_shape& s, const void* X, const floa
       route_dx_kernel<float><<<(unsigned)((tokens + kDxTok - 1) / kDxTok), 256, dx_smem_bytes, st>>>(
           dr, Wr, static_cast<float*>(dX), tokens, s.C, s.M);
     }
-    route_dw_partial_kernel<float><<<wgrid, 256, 0, st>>>(static_cast<const float*>(X), dr, part, tokens, s.C, s.M);
+    launch_dw_partial(static_cast<const float*>(X), dr, part, tokens, s.C, s.M, wgrid, st);
   }
   MOGA_CUDA_OK(cudaGetLastError());
   route_dw_reduce_kernel<<<64, 256, 0, st>>>(part, dWr, colsum, dbias, s.C, s.M, nblk);
