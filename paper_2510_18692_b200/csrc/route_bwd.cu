@@ -130,6 +130,18 @@ __device__ __forceinline__ void store4(__nv_bfloat16* p, const float (&v)[4]) {
   *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
 }
 
+// WT[i, c] = W[c, i]: the dX kernel stages chunks of 128 channels of every logit column, which are
+// contiguous in this order (read from W itself they were 4-byte pieces M floats apart, and the staging took
+// longer than the products).
+__global__ void __launch_bounds__(256)
+route_wt_kernel(const float* __restrict__ Wr, float* __restrict__ WT, int C, int M) {
+  const long long n = (long long)C * M;
+  for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < n; idx += (long long)gridDim.x * blockDim.x) {
+    const int i = (int)(idx / C), c = (int)(idx % C);
+    WT[idx] = Wr[(size_t)c * M + i];
+  }
+}
+
 // dX[t, c] = sum_i dr[t, i] W[c, i].  Block: 64 tokens, all channels in chunks of 128.  Thread
 // (lane = channel quad, warp = token octet) owns 8 tokens x 4 channels; per logit column it reads
 // two 16-byte words of dr (the same for the whole warp) and one of W, for 32 multiply-adds.
@@ -137,7 +149,7 @@ __device__ __forceinline__ void store4(__nv_bfloat16* p, const float (&v)[4]) {
 constexpr int kDxTok = 64, kDxCh = 128;
 template <typename XT>
 __global__ void __launch_bounds__(256)
-route_dx_kernel(const float* __restrict__ dr, const float* __restrict__ Wr, XT* __restrict__ dX, long long tokens, int C,
+route_dx_kernel(const float* __restrict__ dr, const float* __restrict__ WT, XT* __restrict__ dX, long long tokens, int C,
                 int M) {
   extern __shared__ __align__(16) float dx_smem[];
   float* drT = dx_smem;                   // [M][kDxTok]
@@ -152,7 +164,7 @@ route_dx_kernel(const float* __restrict__ dr, const float* __restrict__ Wr, XT* 
     __syncthreads();
     for (int idx = threadIdx.x; idx < kDxCh * M; idx += 256) {
       const int i = idx / kDxCh, cc = idx % kDxCh;        // consecutive threads: consecutive channels
-      wT[i * kDxCh + cc] = c0 + cc < C ? Wr[(size_t)(c0 + cc) * M + i] : 0.f;
+      wT[i * kDxCh + cc] = c0 + cc < C ? WT[(size_t)i * C + c0 + cc] : 0.f;
     }
     __syncthreads();
     float acc[8][4];
@@ -313,13 +325,18 @@ moga_status launch_route_backward(const moga_shape& s, const void* X, const floa
   route_dlogits_kernel<<<nblk, kDrThreads, 0, st>>>(logits, gid, dgate, dr, colsum, tokens, s.M, s.k, s.gate_mode);
   MOGA_CUDA_OK(cudaGetLastError());
   dim3 wgrid((s.C + kWcChunk - 1) / kWcChunk, kSlabs);
+  if (dX) {
+    // W transposed, in the head of the partial-sum scratch: the dW_r kernel writes that scratch after the dX kernel has run
+    route_wt_kernel<<<64, 256, 0, st>>>(Wr, part, s.C, s.M);
+    MOGA_CUDA_OK(cudaGetLastError());
+  }
   const size_t dx_smem_bytes = sizeof(float) * (size_t)s.M * (kDxTok + kDxCh);
   if (s.dtype == MOGA_BF16) {
     if (dX) {
       MOGA_CUDA_OK(cudaFuncSetAttribute(route_dx_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)(sizeof(float) * kMaxM * (kDxTok + kDxCh))));
       route_dx_kernel<__nv_bfloat16><<<(unsigned)((tokens + kDxTok - 1) / kDxTok), 256, dx_smem_bytes, st>>>(
-          dr, Wr, static_cast<__nv_bfloat16*>(dX), tokens, s.C, s.M);
+          dr, part, static_cast<__nv_bfloat16*>(dX), tokens, s.C, s.M);
     }
     launch_dw_partial(static_cast<const __nv_bfloat16*>(X), dr, part, tokens, s.C, s.M, wgrid, st);
   } else {
@@ -327,7 +344,7 @@ moga_status launch_route_backward(const moga_shape& s, const void* X, const floa
       MOGA_CUDA_OK(cudaFuncSetAttribute(route_dx_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)(sizeof(float) * kMaxM * (kDxTok + kDxCh))));
       route_dx_kernel<float><<<(unsigned)((tokens + kDxTok - 1) / kDxTok), 256, dx_smem_bytes, st>>>(
-          dr, Wr, static_cast<float*>(dX), tokens, s.C, s.M);
+          dr, part, static_cast<float*>(dX), tokens, s.C, s.M);
     }
     launch_dw_partial(static_cast<const float*>(X), dr, part, tokens, s.C, s.M, wgrid, st);
   }
