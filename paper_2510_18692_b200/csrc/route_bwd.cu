@@ -18,18 +18,6 @@ constexpr int kDrThreads = 128;       // tokens per block of the dr kernel
 constexpr int kSlabs = 32;            // token slabs of the dW_r partial sums
 constexpr int kWcChunk = 128;         // channels per block of the dW_r kernel
 
-template <typename XT>
-__device__ __forceinline__ float to_f32(XT v);
-template <>
-__device__ __forceinline__ float to_f32<float>(float v) { return v; }
-template <>
-__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
-template <typename XT>
-__device__ __forceinline__ XT from_f32(float v);
-template <>
-__device__ __forceinline__ float from_f32<float>(float v) { return v; }
-template <>
-__device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
 // dr[t, 0..M) for token t = blockIdx.x * 128 + threadIdx.x (tokens of all batch items in one list),
 // and colsum[blockIdx.x, i] = sum of dr[., i] over the block's tokens, added in thread order.
