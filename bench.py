@@ -40,7 +40,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes of the attention kernel / its algorithmic bytes, from the ncu capture of the
 # clip-sized case (traffic grows with T*H: every Q/K/V/O byte crosses DRAM once).  The figure
 # belongs to one version of the kernel source: when the source's hash differs, traffic is null.
-ATTN_TRAFFIC = {"duo": {"file": "attn_bf16_duo.cu", "ratio": 0.9578, "source_sha16": "1e38bd7277bef42b"},
+ATTN_TRAFFIC = {"duo": {"file": "attn_bf16_duo.cu", "ratio": 0.9574, "source_sha16": "efd7d44a4d983365"},
                 "single": {"file": "attn_bf16.cu", "ratio": 0.9565, "source_sha16": "6a7a8dee240eb5b1"}}
 
 
